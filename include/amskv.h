@@ -1,0 +1,211 @@
+/*
+ * amskv.h -- C ABI of the AMS-KV hot path on one NVIDIA B200 (sm_100a).
+ *
+ * What the library does (AMS-KV, "Adaptive Multi-Scale KV Caching", Sec. 4.3):
+ * a next-scale-prediction transformer generates an image scale by scale; the keys and
+ * values of every finished scale are cached per layer.  This library owns that cache as
+ * one segment per scale, keeps only the segments the policy retains (the condensed,
+ * coarsest scales plus the most recent, local scales in cache-efficient layers; every
+ * scale in cache-demanding layers), and computes exact softmax attention of the current
+ * scale's queries over exactly the retained segments.
+ *
+ * Conventions
+ *  - Scales are numbered from 0.  A scale of side s has s*s tokens in row-major raster
+ *    order (token = y*s + x).  rows = 2 * batch when classifier-free guidance doubles it.
+ *  - Every function returns AMSKV_OK (0) or a negative AMSKV_ERR_* code.  Nothing throws,
+ *    aborts or prints.
+ *  - "device pointer" = memory of the current CUDA device, owned by the caller, bf16 unless
+ *    said otherwise, innermost (channel) dimension contiguous, 16-byte aligned, and valid
+ *    until the stream has executed the call.  "host pointer" = ordinary host memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *  - amskv_append / amskv_attend / amskv_layer_similarity only enqueue work on `stream`:
+ *    they allocate nothing, copy nothing between host and device and do not synchronise.
+ *  - A cache object may be used by one host thread at a time.
+ *  - There is no CPU implementation behind any entry point: without a CUDA device the
+ *    compute calls fail with AMSKV_ERR_CUDA.
+ */
+#ifndef AMSKV_H_
+#define AMSKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define AMSKV_API __attribute__((visibility("default")))
+#else
+#define AMSKV_API
+#endif
+
+#define AMSKV_OK 0
+#define AMSKV_ERR_INVALID (-1)        /* bad argument (null, out of range, misaligned)      */
+#define AMSKV_ERR_ORDER (-2)          /* call out of the append/attend order contract       */
+#define AMSKV_ERR_NOMEM (-3)          /* arena too small or device allocation failed         */
+#define AMSKV_ERR_UNSUPPORTED (-4)    /* shape or mode this build does not handle            */
+#define AMSKV_ERR_CUDA (-5)           /* a CUDA runtime / driver call failed                 */
+#define AMSKV_ERR_DEVICE_TIMEOUT (-6) /* a bounded device-side wait gave up (see amskv_status) */
+
+#define AMSKV_MAX_SCALES 32
+
+/* amskv_desc.flags */
+#define AMSKV_FLAG_PLAN_ONLY 1u /* host bookkeeping only: no device memory is touched and
+                                   attend / similarity are refused; append takes NULL K, V.
+                                   For sizing and for inspecting the policy without a GPU. */
+
+/* amskv_set_attend_path */
+#define AMSKV_PATH_AUTO 0   /* small-query kernel for few query tokens, tensor cores otherwise */
+#define AMSKV_PATH_SIMT 1   /* always the CUDA-core kernel                                     */
+#define AMSKV_PATH_TENSOR 2 /* always the tcgen05 kernel                                       */
+
+typedef struct amskv_cache amskv_cache; /* opaque; owned by the library */
+
+/*
+ * Per-layer policy (Sec. 4.1 scale groups, Sec. 4.2 layer classes).
+ *   n_condensed      c >= 0: the first c scales are pinned (the paper's C_cds, counted in
+ *                    scales; the ablation in Appendix A uses 0, 1 and 2).
+ *   n_local          w >= 1: the w most recent scales are kept, the just-appended one
+ *                    included (Algorithm 2 keeps the tail of the cache after the append).
+ *   cache_demanding  non-zero: the layer keeps every scale (full retention).
+ * A cache-efficient layer keeps scale s at step k iff s < c or s > k - w.
+ */
+typedef struct {
+    int32_t n_condensed;
+    int32_t n_local;
+    int32_t cache_demanding;
+} amskv_layer_policy;
+
+typedef struct {
+    int32_t layers;
+    int32_t heads;
+    int32_t head_dim;            /* 64 or 128                                              */
+    int32_t rows;                /* sequences held at once (2 * batch under guidance)      */
+    int32_t n_scales;            /* 1 .. AMSKV_MAX_SCALES                                  */
+    const int32_t* scale_sides;  /* [n_scales] side lengths, each >= 1; copied             */
+    const amskv_layer_policy* policy; /* [layers]; copied                                  */
+    float softmax_scale;         /* <= 0 selects 1/sqrt(head_dim)                          */
+    uint32_t flags;              /* AMSKV_FLAG_*                                           */
+} amskv_desc;
+
+/* Bytes of device memory a cache for `desc` needs (its KV arena; Appendix D, Eq. 5 counts
+ * the same tokens).  Host-only. */
+AMSKV_API int amskv_cache_required_bytes(const amskv_desc* desc, size_t* bytes);
+
+/*
+ * Create a cache (one independent cache per layer, Sec. 4.3).
+ *   dev_mem    device pointer to an arena of dev_bytes bytes, 256-byte aligned, owned by the
+ *              caller and kept alive until destroy; or NULL, in which case the library
+ *              allocates (and later frees) the arena itself.
+ * The arena is zero-filled on the default stream and the call synchronises once.
+ * Errors: INVALID (descriptor), NOMEM (dev_bytes too small, allocation failed), CUDA.
+ */
+AMSKV_API int amskv_cache_create(const amskv_desc* desc, void* dev_mem, size_t dev_bytes, amskv_cache** out);
+
+/* Free the object, and the arena only if the library allocated it. */
+AMSKV_API int amskv_cache_destroy(amskv_cache* cache);
+
+/* Forget all appended scales (start a new batch of images).  Metadata only. */
+AMSKV_API int amskv_cache_reset(amskv_cache* cache);
+
+/*
+ * Append scale `scale` of `layer` and evict in place (Algorithm 1 "append", then
+ * Algorithm 2 "rolling", at scale granularity).
+ *   K, V      device pointers, logical shape [rows, heads, T, head_dim], T = side^2.
+ *   strides   element strides of the (row, head, token) dimensions, or NULL for a
+ *             contiguous tensor; the token and head strides must be multiples of 8.
+ * The segment that leaves the local window is dropped by bookkeeping alone; its slot is
+ * the one the new segment is written to.  Scales must be appended in order 0, 1, 2, ...
+ * per layer (ORDER otherwise).  Non-finite K/V values give unspecified results.
+ */
+AMSKV_API int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const void* V,
+                 const int64_t strides[3], void* stream);
+
+/*
+ * Attention of the queries of `scale` over the segments `layer` retains at that step
+ * (Sec. 3.1, Eq. 2: a whole scale is conditioned on whole earlier scales, so there is no
+ * mask inside the retained set):  out = softmax(softmax_scale * Q K^T) V.
+ *   Q, out    device pointers, [rows, heads, T, head_dim] bf16; strides as in append.
+ * `scale` must be the scale most recently appended to `layer` (ORDER otherwise).
+ * Arithmetic: bf16 inputs, fp32 accumulation, probabilities rounded to bf16 before the
+ * second product on the tensor-core path, bf16 output.
+ */
+AMSKV_API int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* out,
+                 const int64_t q_strides[3], const int64_t o_strides[3], void* stream);
+
+/* Choose the kernel used by amskv_attend (AMSKV_PATH_*).  The default is AUTO. */
+AMSKV_API int amskv_set_attend_path(amskv_cache* cache, int path);
+
+/*
+ * One generation step from HOST buffers: copies K, V, Q of `scale` (contiguous
+ * [rows, heads, T, head_dim] bf16 host arrays; pinned memory makes the copies asynchronous)
+ * into `staging`, appends, attends and copies the result to the host array `out`.
+ *   staging        device pointer, at least amskv_step_staging_bytes() bytes, 256-byte aligned.
+ * Everything is enqueued on `stream`; the host arrays must stay valid until it has run.
+ */
+AMSKV_API int amskv_step_host(amskv_cache* cache, int layer, int scale, const void* K_host, const void* V_host,
+                    const void* Q_host, void* out_host, void* staging, size_t staging_bytes,
+                    void* stream);
+
+/* Bytes of staging amskv_step_host needs for the largest scale of this cache. */
+AMSKV_API int amskv_step_staging_bytes(const amskv_cache* cache, size_t* bytes);
+
+/*
+ * Inter-scale key similarity (Sec. 4.3, Eq. 4): resizes the keys of the previous scale to
+ * the current scale's side by 2-D bilinear interpolation (half-pixel centres, edge clamp)
+ * and returns the sum over every (row, head, token, channel) of the squared difference,
+ *   ss = || k_i - resize(k_{i-1}) ||_2^2,   so that S = -sqrt(ss).
+ *   K_prev, K_cur   device pointers, contiguous [rows, heads, side^2, head_dim] bf16.
+ *   out_ss          device pointer to one double (written by the kernel).
+ *   workspace       device pointer, amskv_similarity_workspace_bytes() bytes, 256-byte
+ *                   aligned; scratch for per-block partial sums, overwritten by every call,
+ *                   so calls sharing a workspace must not overlap on the device.
+ * The reduction order is fixed, so equal inputs give bit-equal results.
+ */
+AMSKV_API int amskv_layer_similarity(const void* K_prev, int side_prev, const void* K_cur, int side_cur,
+                           int rows, int heads, int head_dim, double* out_ss, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
+/* Bytes of workspace amskv_layer_similarity needs (independent of the problem size). */
+AMSKV_API size_t amskv_similarity_workspace_bytes(void);
+
+/*
+ * Layer classification from similarity scores (host-only).
+ *   by threshold: demanding[l] = scores[l] < theta (strict; Algorithm 1).
+ *   by rank:      the n_demanding lowest-scoring layers are demanding, ties to the lower
+ *                 layer index (the similarity-aware allocation S2 of Sec. 4.2).
+ */
+AMSKV_API int amskv_classify_by_threshold(const double* scores, int layers, double theta, int32_t* demanding);
+AMSKV_API int amskv_classify_lowest(const double* scores, int layers, int n_demanding, int32_t* demanding);
+
+/* Segment ids `layer` retains right after scale `scale` was appended, ascending (host-only;
+ * a pure function of the policy).  ids must hold AMSKV_MAX_SCALES entries. */
+AMSKV_API int amskv_kept_segments(const amskv_cache* cache, int layer, int scale, int32_t* ids, int32_t* n);
+
+/* Segment ids the append of `scale` drops from `layer` (host-only). */
+AMSKV_API int amskv_evicted_at(const amskv_cache* cache, int layer, int scale, int32_t* ids, int32_t* n);
+
+/* Token ranges (start, length) of the layer's per-(row, head) arena region that attend
+ * reads at `scale`, merged where adjacent (host-only).  ranges must hold
+ * 2 * AMSKV_MAX_SCALES entries. */
+AMSKV_API int amskv_resident_ranges(const amskv_cache* cache, int layer, int scale, int32_t* ranges, int32_t* n);
+
+/* Bytes: the arena, the KV bytes resident now, and the largest residency seen since the
+ * last reset. */
+AMSKV_API int amskv_cache_bytes(const amskv_cache* cache, size_t* allocated, size_t* resident_now, size_t* peak);
+
+/* Reads the device status word (synchronises the device).  *device_status is 0 when no
+ * kernel reported a problem; otherwise the code of the first bounded wait that gave up, and
+ * the return value is AMSKV_ERR_DEVICE_TIMEOUT. */
+AMSKV_API int amskv_status(amskv_cache* cache, int* device_status);
+
+/* Number of kernels this library has launched since it was loaded. */
+AMSKV_API int64_t amskv_launch_count(void);
+
+AMSKV_API const char* amskv_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMSKV_H_ */

@@ -1,0 +1,424 @@
+// C ABI of the AMS-KV library: argument checking, the segment table and kernel launches.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <numeric>
+#include <vector>
+
+#include "../../include/amskv.h"
+#include "kernels.cuh"
+
+namespace amskv {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+constexpr size_t kAlign = 256;
+constexpr size_t kStatusBytes = 256;
+constexpr int kSmallQueryMaxTokens = 16;  // scales with at most this many query tokens use the CUDA-core kernel
+
+static size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct alignas(64) TensorMapBlob {
+    unsigned char bytes[128];
+};
+
+}  // namespace amskv
+
+using namespace amskv;
+
+struct amskv_cache {
+    int32_t layers = 0, heads = 0, head_dim = 0, rows = 0, n_scales = 0;
+    uint32_t flags = 0;
+    float softmax_scale = 0.f;
+    int path = AMSKV_PATH_AUTO;
+    int sm_count = 0;
+    std::vector<int32_t> sides, tokens;
+    std::vector<LayerLayout> layout;
+    std::vector<size_t> layer_offset;  // bytes from the arena start
+    std::vector<int32_t> last_appended;
+    std::vector<TensorMapBlob> k_maps, v_maps;
+    bool tc_ready = false;
+    char* arena = nullptr;
+    size_t arena_bytes = 0;
+    bool owns_arena = false;
+    size_t resident_now = 0, peak = 0;
+
+    bool plan_only() const { return (flags & AMSKV_FLAG_PLAN_ONLY) != 0; }
+    int64_t items() const { return (int64_t)rows * heads; }
+    size_t token_bytes() const { return (size_t)items() * head_dim * 2 /*bf16*/ * 2 /*K and V*/; }
+    LayerRegion region(int layer) const
+    {
+        return LayerRegion{reinterpret_cast<__nv_bfloat16*>(arena + layer_offset[layer]), layout[layer].capacity};
+    }
+    int* status_word() const { return reinterpret_cast<int*>(arena); }
+};
+
+namespace {
+
+int check_desc(const amskv_desc* d)
+{
+    if (!d || !d->scale_sides || !d->policy) return AMSKV_ERR_INVALID;
+    if (d->layers < 1 || d->heads < 1 || d->rows < 1) return AMSKV_ERR_INVALID;
+    if (d->n_scales < 1 || d->n_scales > AMSKV_MAX_SCALES) return AMSKV_ERR_INVALID;
+    if (d->head_dim != 64 && d->head_dim != 128) return AMSKV_ERR_UNSUPPORTED;
+    for (int i = 0; i < d->n_scales; ++i)
+        if (d->scale_sides[i] < 1 || d->scale_sides[i] > 4096) return AMSKV_ERR_INVALID;
+    for (int l = 0; l < d->layers; ++l)
+        if (d->policy[l].n_condensed < 0 || d->policy[l].n_local < 1) return AMSKV_ERR_INVALID;
+    if ((d->flags & ~AMSKV_FLAG_PLAN_ONLY) != 0) return AMSKV_ERR_INVALID;
+    if (!(d->softmax_scale == d->softmax_scale)) return AMSKV_ERR_INVALID;  // NaN
+    return AMSKV_OK;
+}
+
+// Fills everything that depends only on the descriptor.
+int plan(const amskv_desc* d, amskv_cache* c)
+{
+    c->layers = d->layers;
+    c->heads = d->heads;
+    c->head_dim = d->head_dim;
+    c->rows = d->rows;
+    c->n_scales = d->n_scales;
+    c->flags = d->flags;
+    c->softmax_scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / std::sqrt((float)d->head_dim);
+    c->sides.assign(d->scale_sides, d->scale_sides + d->n_scales);
+    c->tokens.resize(d->n_scales);
+    for (int i = 0; i < d->n_scales; ++i) {
+        const int64_t t = (int64_t)c->sides[i] * c->sides[i];
+        if (t > (1 << 24)) return AMSKV_ERR_INVALID;
+        c->tokens[i] = (int32_t)t;
+    }
+    c->layout.resize(d->layers);
+    c->layer_offset.resize(d->layers);
+    size_t at = kStatusBytes;
+    for (int l = 0; l < d->layers; ++l) {
+        c->layout[l].build(c->tokens, d->policy[l].n_condensed, d->policy[l].n_local, d->policy[l].cache_demanding != 0);
+        if ((int64_t)c->layout[l].capacity > (1ll << 30)) return AMSKV_ERR_INVALID;
+        c->layer_offset[l] = at;
+        at += align_up((size_t)c->layout[l].capacity * c->token_bytes());
+    }
+    c->arena_bytes = at;
+    c->last_appended.assign(d->layers, -1);
+    return AMSKV_OK;
+}
+
+bool bad_layer_scale(const amskv_cache* c, int layer, int scale)
+{
+    return !c || layer < 0 || layer >= c->layers || scale < 0 || scale >= c->n_scales;
+}
+
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+int make_strided(const void* ptr, const int64_t* strides, int32_t heads, int32_t T, int32_t D, Strided* out)
+{
+    if (!ptr || misaligned(ptr)) return AMSKV_ERR_INVALID;
+    out->ptr = ptr;
+    if (strides) {
+        out->row = strides[0];
+        out->head = strides[1];
+        out->token = strides[2];
+        if (out->row < 0 || out->head < 0 || out->token < D) return AMSKV_ERR_INVALID;
+        if ((out->row % 8) || (out->head % 8) || (out->token % 8)) return AMSKV_ERR_INVALID;
+    } else {
+        out->token = D;
+        out->head = (int64_t)T * D;
+        out->row = (int64_t)heads * T * D;
+    }
+    return AMSKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int amskv_cache_required_bytes(const amskv_desc* desc, size_t* bytes)
+{
+    if (!bytes) return AMSKV_ERR_INVALID;
+    int rc = check_desc(desc);
+    if (rc != AMSKV_OK) return rc;
+    amskv_cache tmp;
+    rc = plan(desc, &tmp);
+    if (rc != AMSKV_OK) return rc;
+    *bytes = tmp.arena_bytes;
+    return AMSKV_OK;
+}
+
+int amskv_cache_create(const amskv_desc* desc, void* dev_mem, size_t dev_bytes, amskv_cache** out)
+{
+    if (!out) return AMSKV_ERR_INVALID;
+    *out = nullptr;
+    int rc = check_desc(desc);
+    if (rc != AMSKV_OK) return rc;
+    amskv_cache* c = new (std::nothrow) amskv_cache();
+    if (!c) return AMSKV_ERR_NOMEM;
+    rc = plan(desc, c);
+    if (rc != AMSKV_OK) { delete c; return rc; }
+    if (c->plan_only()) { *out = c; return AMSKV_OK; }
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete c;
+        return AMSKV_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+    if (dev_mem) {
+        if ((reinterpret_cast<uintptr_t>(dev_mem) % kAlign) != 0) { delete c; return AMSKV_ERR_INVALID; }
+        if (dev_bytes < c->arena_bytes) { delete c; return AMSKV_ERR_NOMEM; }
+        c->arena = static_cast<char*>(dev_mem);
+    } else {
+        size_t free_b = 0, total_b = 0;
+        if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) { (void)cudaGetLastError(); delete c; return AMSKV_ERR_CUDA; }
+        if (free_b < c->arena_bytes) { delete c; return AMSKV_ERR_NOMEM; }
+        void* p = nullptr;
+        if (cudaMalloc(&p, c->arena_bytes) != cudaSuccess) { (void)cudaGetLastError(); delete c; return AMSKV_ERR_NOMEM; }
+        c->arena = static_cast<char*>(p);
+        c->owns_arena = true;
+    }
+    // Tiles may extend past a range's end into tokens nobody attends; zero-filling once keeps
+    // those bytes finite so that a zero probability times such a value is zero.
+    cudaError_t e = cudaMemsetAsync(c->arena, 0, c->arena_bytes, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        if (c->owns_arena) cudaFree(c->arena);
+        delete c;
+        return AMSKV_ERR_CUDA;
+    }
+    c->tc_ready = false;
+    if (tc_supported(c->head_dim) && prop.major == 10) {
+        c->k_maps.resize(c->layers);
+        c->v_maps.resize(c->layers);
+        bool ok = true;
+        for (int l = 0; l < c->layers && ok; ++l)
+            ok = tc_encode_kv_maps(c->region(l), c->items(), c->head_dim, c->k_maps[l].bytes, c->v_maps[l].bytes);
+        c->tc_ready = ok;
+    }
+    *out = c;
+    return AMSKV_OK;
+}
+
+int amskv_cache_destroy(amskv_cache* cache)
+{
+    if (!cache) return AMSKV_ERR_INVALID;
+    int rc = AMSKV_OK;
+    if (cache->owns_arena && cache->arena) {
+        if (cudaFree(cache->arena) != cudaSuccess) { (void)cudaGetLastError(); rc = AMSKV_ERR_CUDA; }
+    }
+    delete cache;
+    return rc;
+}
+
+int amskv_cache_reset(amskv_cache* cache)
+{
+    if (!cache) return AMSKV_ERR_INVALID;
+    std::fill(cache->last_appended.begin(), cache->last_appended.end(), -1);
+    cache->resident_now = 0;
+    cache->peak = 0;
+    return AMSKV_OK;
+}
+
+int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const void* V, const int64_t strides[3],
+                 void* stream)
+{
+    if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
+    const int32_t T = cache->tokens[scale];
+    const LayerLayout& lay = cache->layout[layer];
+    if (!cache->plan_only()) {
+        Strided ks, vs;
+        int rc = make_strided(K, strides, cache->heads, T, cache->head_dim, &ks);
+        if (rc != AMSKV_OK) return rc;
+        rc = make_strided(V, strides, cache->heads, T, cache->head_dim, &vs);
+        if (rc != AMSKV_OK) return rc;
+        cudaError_t e = launch_append(ks, vs, cache->region(layer), lay.offset[scale], T, cache->rows, cache->heads,
+                                      cache->head_dim, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    }
+    const int64_t before = scale > 0 ? lay.resident_tokens(cache->tokens, scale - 1) : 0;
+    const int64_t after = lay.resident_tokens(cache->tokens, scale);
+    cache->resident_now = (size_t)((int64_t)cache->resident_now + (after - before) * (int64_t)cache->token_bytes());
+    cache->peak = std::max(cache->peak, cache->resident_now);
+    cache->last_appended[layer] = scale;
+    return AMSKV_OK;
+}
+
+int amskv_set_attend_path(amskv_cache* cache, int path)
+{
+    if (!cache || path < AMSKV_PATH_AUTO || path > AMSKV_PATH_TENSOR) return AMSKV_ERR_INVALID;
+    if (path == AMSKV_PATH_TENSOR && !cache->tc_ready) return AMSKV_ERR_UNSUPPORTED;
+    cache->path = path;
+    return AMSKV_OK;
+}
+
+int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* out, const int64_t q_strides[3],
+                 const int64_t o_strides[3], void* stream)
+{
+    if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
+    if (scale != cache->last_appended[layer]) return AMSKV_ERR_ORDER;
+    const int32_t T = cache->tokens[scale];
+    Strided q, o;
+    int rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
+    if (rc != AMSKV_OK) return rc;
+    rc = make_strided(out, o_strides, cache->heads, T, cache->head_dim, &o);
+    if (rc != AMSKV_OK) return rc;
+    RangeList ranges;
+    ranges.n = cache->layout[layer].ranges(cache->tokens, scale, ranges.r);
+    ranges.total = 0;
+    for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
+    bool tensor = cache->path == AMSKV_PATH_TENSOR ||
+                  (cache->path == AMSKV_PATH_AUTO && cache->tc_ready && T > kSmallQueryMaxTokens);
+    cudaError_t e;
+    if (tensor) {
+        e = launch_attend_tc(q, o, cache->region(layer), cache->k_maps[layer].bytes, cache->v_maps[layer].bytes, ranges,
+                             T, cache->rows, cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
+                             cache->sm_count, static_cast<cudaStream_t>(stream));
+    } else {
+        e = launch_attend_simt(q, o, cache->region(layer), ranges, T, cache->rows, cache->heads, cache->head_dim,
+                               cache->softmax_scale, static_cast<cudaStream_t>(stream));
+    }
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
+}
+
+int amskv_step_staging_bytes(const amskv_cache* cache, size_t* bytes)
+{
+    if (!cache || !bytes) return AMSKV_ERR_INVALID;
+    const int32_t tmax = *std::max_element(cache->tokens.begin(), cache->tokens.end());
+    const size_t one = align_up((size_t)cache->items() * tmax * cache->head_dim * 2);
+    *bytes = 4 * one;  // K, V, Q, out
+    return AMSKV_OK;
+}
+
+int amskv_step_host(amskv_cache* cache, int layer, int scale, const void* K_host, const void* V_host,
+                    const void* Q_host, void* out_host, void* staging, size_t staging_bytes, void* stream)
+{
+    if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
+    if (!K_host || !V_host || !Q_host || !out_host || !staging) return AMSKV_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(staging) % kAlign) != 0) return AMSKV_ERR_INVALID;
+    size_t need = 0;
+    amskv_step_staging_bytes(cache, &need);
+    if (staging_bytes < need) return AMSKV_ERR_NOMEM;
+    if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
+    const size_t one = need / 4;
+    const size_t bytes = (size_t)cache->items() * cache->tokens[scale] * cache->head_dim * 2;
+    char* s = static_cast<char*>(staging);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(s, K_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s + one, V_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s + 2 * one, Q_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    int rc = amskv_append(cache, layer, scale, s, s + one, nullptr, stream);
+    if (rc != AMSKV_OK) return rc;
+    rc = amskv_attend(cache, layer, scale, s + 2 * one, s + 3 * one, nullptr, nullptr, stream);
+    if (rc != AMSKV_OK) return rc;
+    e = cudaMemcpyAsync(out_host, s + 3 * one, bytes, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
+}
+
+size_t amskv_similarity_workspace_bytes(void) { return align_up(sizeof(double) * kSimilarityMaxBlocks); }
+
+int amskv_layer_similarity(const void* K_prev, int side_prev, const void* K_cur, int side_cur, int rows, int heads,
+                           int head_dim, double* out_ss, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!K_prev || !K_cur || !out_ss || !workspace) return AMSKV_ERR_INVALID;
+    if (misaligned(K_prev) || misaligned(K_cur) || (reinterpret_cast<uintptr_t>(out_ss) & 7u)) return AMSKV_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return AMSKV_ERR_INVALID;
+    if (side_prev < 1 || side_cur < 1 || side_prev > 4096 || side_cur > 4096 || rows < 1 || heads < 1)
+        return AMSKV_ERR_INVALID;
+    if (head_dim != 64 && head_dim != 128) return AMSKV_ERR_UNSUPPORTED;
+    if (workspace_bytes < amskv_similarity_workspace_bytes()) return AMSKV_ERR_NOMEM;
+    cudaError_t e = launch_similarity((const __nv_bfloat16*)K_prev, side_prev, (const __nv_bfloat16*)K_cur, side_cur,
+                                      (int64_t)rows * heads, head_dim, out_ss, static_cast<double*>(workspace),
+                                      static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
+}
+
+int amskv_classify_by_threshold(const double* scores, int layers, double theta, int32_t* demanding)
+{
+    if (!scores || !demanding || layers < 1) return AMSKV_ERR_INVALID;
+    for (int l = 0; l < layers; ++l) demanding[l] = scores[l] < theta ? 1 : 0;
+    return AMSKV_OK;
+}
+
+int amskv_classify_lowest(const double* scores, int layers, int n_demanding, int32_t* demanding)
+{
+    if (!scores || !demanding || layers < 1 || n_demanding < 0 || n_demanding > layers) return AMSKV_ERR_INVALID;
+    std::vector<int> order(layers);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return scores[a] < scores[b]; });
+    for (int l = 0; l < layers; ++l) demanding[l] = 0;
+    for (int i = 0; i < n_demanding; ++i) demanding[order[i]] = 1;
+    return AMSKV_OK;
+}
+
+int amskv_kept_segments(const amskv_cache* cache, int layer, int scale, int32_t* ids, int32_t* n)
+{
+    if (bad_layer_scale(cache, layer, scale) || !ids || !n) return AMSKV_ERR_INVALID;
+    *n = cache->layout[layer].kept(scale, ids);
+    return AMSKV_OK;
+}
+
+int amskv_evicted_at(const amskv_cache* cache, int layer, int scale, int32_t* ids, int32_t* n)
+{
+    if (bad_layer_scale(cache, layer, scale) || !ids || !n) return AMSKV_ERR_INVALID;
+    *n = cache->layout[layer].evicted(scale, ids);
+    return AMSKV_OK;
+}
+
+int amskv_resident_ranges(const amskv_cache* cache, int layer, int scale, int32_t* ranges, int32_t* n)
+{
+    if (bad_layer_scale(cache, layer, scale) || !ranges || !n) return AMSKV_ERR_INVALID;
+    Range r[kMaxRanges];
+    *n = cache->layout[layer].ranges(cache->tokens, scale, r);
+    for (int i = 0; i < *n; ++i) {
+        ranges[2 * i] = r[i].start;
+        ranges[2 * i + 1] = r[i].len;
+    }
+    return AMSKV_OK;
+}
+
+int amskv_cache_bytes(const amskv_cache* cache, size_t* allocated, size_t* resident_now, size_t* peak)
+{
+    if (!cache) return AMSKV_ERR_INVALID;
+    if (allocated) *allocated = cache->arena_bytes;
+    if (resident_now) *resident_now = cache->resident_now;
+    if (peak) *peak = cache->peak;
+    return AMSKV_OK;
+}
+
+int amskv_status(amskv_cache* cache, int* device_status)
+{
+    if (!cache || !device_status) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) { *device_status = 0; return AMSKV_OK; }
+    int word = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&word, cache->status_word(), sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    *device_status = word;
+    return word == 0 ? AMSKV_OK : AMSKV_ERR_DEVICE_TIMEOUT;
+}
+
+int64_t amskv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* amskv_strerror(int code)
+{
+    switch (code) {
+        case AMSKV_OK: return "ok";
+        case AMSKV_ERR_INVALID: return "invalid argument";
+        case AMSKV_ERR_ORDER: return "call out of order";
+        case AMSKV_ERR_NOMEM: return "not enough device memory";
+        case AMSKV_ERR_UNSUPPORTED: return "unsupported shape or mode";
+        case AMSKV_ERR_CUDA: return "CUDA call failed";
+        case AMSKV_ERR_DEVICE_TIMEOUT: return "a device-side wait gave up";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,67 @@
+// Internal interface between the C ABI (api.cu) and the kernels.  Not installed.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "policy.hpp"
+
+namespace amskv {
+
+constexpr int kMaxRanges = 32;
+
+// Token ranges of one layer's per-item region that an attention call reads; passed by value.
+struct RangeList {
+    int32_t n;
+    int32_t total;  // sum of len
+    Range r[kMaxRanges];
+};
+
+// A [rows, heads, tokens, D] bf16 tensor described by element strides (D contiguous).
+struct Strided {
+    const void* ptr;
+    int64_t row, head, token;
+};
+
+// One layer's KV region: item i (= row * heads + head) owns 2 * capacity * D bf16 values,
+// keys first ([capacity][D]) and values right behind them.
+struct LayerRegion {
+    __nv_bfloat16* base;
+    int32_t capacity;  // tokens per item
+};
+
+// Device status codes written (first one wins) when a bounded wait gives up.
+enum DeviceStatus : int {
+    kStatusOk = 0,
+    kStatusTmaTimeout = 1,
+    kStatusMmaTimeout = 2,
+    kStatusSyncTimeout = 3,
+    kStatusTmemAlloc = 4,
+};
+
+cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion& region, int32_t token_offset,
+                          int32_t T, int32_t rows, int32_t heads, int32_t D, cudaStream_t stream);
+
+cudaError_t launch_attend_simt(const Strided& Q, const Strided& O, const LayerRegion& region, const RangeList& ranges,
+                               int32_t T, int32_t rows, int32_t heads, int32_t D, float softmax_scale,
+                               cudaStream_t stream);
+
+constexpr int kSimilarityMaxBlocks = 2048;
+cudaError_t launch_similarity(const __nv_bfloat16* K_prev, int32_t side_prev, const __nv_bfloat16* K_cur,
+                              int32_t side_cur, int64_t items, int32_t D, double* out_ss, double* partials,
+                              cudaStream_t stream);
+
+// Tensor-core path.  The tensor maps are built on the host by the caller of launch_attend_tc.
+struct TcMaps;  // defined in attend_tc.cu
+bool tc_supported(int32_t D);
+// Encodes the tensor maps a layer needs for its K and V streams; returns false on failure.
+bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, void* k_map_out, void* v_map_out);
+cudaError_t launch_attend_tc(const Strided& Q, const Strided& O, const LayerRegion& region, const void* k_map,
+                             const void* v_map, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads,
+                             int32_t D, float softmax_scale, int* status, int sm_count, cudaStream_t stream);
+
+void count_launch(int n = 1);
+
+}  // namespace amskv

@@ -1,0 +1,126 @@
+// Inter-scale key similarity (Sec. 4.3, Eq. 4): ss = || k_i - resize(k_{i-1}) ||^2.
+//
+// One thread per (item, output token, 8-channel chunk): it reads 16 bytes of the current
+// scale's keys and the four bilinear neighbours from the previous scale (which is at most as
+// large, so those reads are served by L1/L2 after the first touch), interpolates in fp32 and
+// accumulates the squared differences.  Blocks reduce in fp64 into a partials array; a second
+// single-block kernel adds the partials in a fixed order, so the result is reproducible.
+#include "kernels.cuh"
+
+namespace amskv {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8])
+{
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 v = __bfloat1622float2(h[i]);
+        f[2 * i] = v.x;
+        f[2 * i + 1] = v.y;
+    }
+}
+
+__device__ __forceinline__ double block_sum(double v, double* smem)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) smem[warp] = v;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < kThreads / 32; ++w) total += smem[w];
+    return total;  // valid in thread 0
+}
+
+// source coordinate of output pixel i: (i + 0.5) * s_in / s_out - 0.5, clamped to [0, s_in - 1]
+__device__ __forceinline__ void tap(int i, float ratio, int s_in, int& i0, int& i1, float& w)
+{
+    float f = ((float)i + 0.5f) * ratio - 0.5f;
+    f = fminf(fmaxf(f, 0.f), (float)(s_in - 1));
+    i0 = (int)floorf(f);
+    i1 = min(i0 + 1, s_in - 1);
+    w = f - (float)i0;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+similarity_partial_kernel(const uint4* __restrict__ K_prev, int32_t s_prev, const uint4* __restrict__ K_cur,
+                          int32_t s_cur, int64_t total_chunks, double* __restrict__ partials)
+{
+    constexpr int CPT = D / 8;
+    __shared__ double smem[kThreads / 32];
+    const float ratio = (float)s_prev / (float)s_cur;
+    const int32_t t_cur = s_cur * s_cur, t_prev = s_prev * s_prev;
+    double acc = 0.0;
+    for (int64_t idx = (int64_t)blockIdx.x * kThreads + threadIdx.x; idx < total_chunks;
+         idx += (int64_t)gridDim.x * kThreads) {
+        const int64_t tok_global = idx / CPT;
+        const int32_t ch = (int32_t)(idx - tok_global * CPT);
+        const int64_t item = tok_global / t_cur;
+        const int32_t tok = (int32_t)(tok_global - item * t_cur);
+        const int32_t y = tok / s_cur, x = tok - y * s_cur;
+        int y0, y1, x0, x1;
+        float wy, wx;
+        tap(y, ratio, s_prev, y0, y1, wy);
+        tap(x, ratio, s_prev, x0, x1, wx);
+        const uint4* P = K_prev + item * (int64_t)t_prev * CPT + ch;
+        float c[8], v00[8], v01[8], v10[8], v11[8];
+        unpack8(__ldcs(K_cur + idx), c);
+        unpack8(__ldg(P + (int64_t)(y0 * s_prev + x0) * CPT), v00);
+        unpack8(__ldg(P + (int64_t)(y0 * s_prev + x1) * CPT), v01);
+        unpack8(__ldg(P + (int64_t)(y1 * s_prev + x0) * CPT), v10);
+        unpack8(__ldg(P + (int64_t)(y1 * s_prev + x1) * CPT), v11);
+        float part = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float top = v00[i] + wx * (v01[i] - v00[i]);
+            const float bot = v10[i] + wx * (v11[i] - v10[i]);
+            const float diff = c[i] - (top + wy * (bot - top));
+            part = fmaf(diff, diff, part);
+        }
+        acc += (double)part;
+    }
+    const double total = block_sum(acc, smem);
+    if (threadIdx.x == 0) partials[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(kThreads)
+similarity_final_kernel(const double* __restrict__ partials, int n, double* __restrict__ out)
+{
+    __shared__ double smem[kThreads / 32];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += kThreads) acc += partials[i];
+    const double total = block_sum(acc, smem);
+    if (threadIdx.x == 0) *out = total;
+}
+
+}  // namespace
+
+cudaError_t launch_similarity(const __nv_bfloat16* K_prev, int32_t side_prev, const __nv_bfloat16* K_cur,
+                              int32_t side_cur, int64_t items, int32_t D, double* out_ss, double* partials,
+                              cudaStream_t stream)
+{
+    const int64_t total = items * side_cur * side_cur * (D / 8);
+    int64_t blocks = (total + kThreads - 1) / kThreads;
+    if (blocks > kSimilarityMaxBlocks) blocks = kSimilarityMaxBlocks;
+    if (blocks < 1) blocks = 1;
+    if (D == 64) {
+        similarity_partial_kernel<64><<<(unsigned)blocks, kThreads, 0, stream>>>(
+            (const uint4*)K_prev, side_prev, (const uint4*)K_cur, side_cur, total, partials);
+    } else {
+        similarity_partial_kernel<128><<<(unsigned)blocks, kThreads, 0, stream>>>(
+            (const uint4*)K_prev, side_prev, (const uint4*)K_cur, side_cur, total, partials);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    similarity_final_kernel<<<1, kThreads, 0, stream>>>(partials, (int)blocks, out_ss);
+    count_launch(2);
+    return cudaGetLastError();
+}
+
+}  // namespace amskv
