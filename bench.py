@@ -1,0 +1,458 @@
+#!/usr/bin/env python
+"""Benchmark of the AMS-KV hot path on synthetic VAR-shaped data.
+
+One step = one pass of the whole path over one batch: for every scale, for every layer,
+amskv_append then amskv_attend (the self-attention work of generating one batch of images).
+Metric: self-attention microseconds per image over all scales and layers (lower is better),
+with the roofline fraction and the KV-cache bytes beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload var_d30] [--impl ours|reference]
+
+N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "VAR-d30 self-attn us/image (all scales+layers)"
+UNIT = "us/image"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0
+
+# DRAM traffic of the attention kernels per step, from ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload; filled from the summaries under profiles/.
+NCU_TRAFFIC_BYTES_PER_STEP = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS)), "measured"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def _kept(k, c, w, dem):
+    """Segments read at scale k -- used only to count algorithmic bytes for the roofline."""
+    return [s for s in range(k + 1) if dem or s < c or s > k - w]
+
+
+def algorithmic_work(wl, policies):
+    """Per (layer, scale): bytes = Q read + out write + kept K,V read once; flops = 4 T L D per item."""
+    items = wl.rows * wl.heads
+    tok = wl.tokens
+    per = {}
+    for layer, (c, w, dem) in enumerate(policies):
+        for k in range(len(tok)):
+            L = sum(tok[s] for s in _kept(k, c, w, dem))
+            per[(layer, k)] = (2 * wl.head_dim * items * (2 * tok[k] + 2 * L), 4 * tok[k] * L * wl.head_dim * items)
+    return per
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2511_16047_b200 import binding as B
+    from paper_2511_16047_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = synth.WORKLOADS[args.workload]
+    if args.batch:
+        wl = wl.replace(batch=args.batch)
+    hbm_gbs, tflops, peak_kind = _peaks()
+    K = len(wl.sides)
+    tok = wl.tokens
+    stream = torch.cuda.current_stream()
+
+    # inputs: one Q/K/V set per scale, shared by the layers (each layer has its own cache region,
+    # so no K/V read by attention is shared between layers)
+    qkv = [synth.qkv_for_scale(wl.rows, wl.heads, tok[k], wl.head_dim, wl.seed, k, "cuda") for k in range(K)]
+    outs = [torch.empty_like(q) for q, _, _ in qkv]
+    input_bytes = sum(3 * q.numel() * 2 for q, _, _ in qkv)
+
+    def measure(policies, label, instrument):
+        desc, keep = B.make_desc(wl.layers, wl.heads, wl.head_dim, wl.rows, wl.sides, policies)
+        nbytes = B.amskv_cache_required_bytes(desc)
+        free_b, _ = torch.cuda.mem_get_info()
+        if nbytes + (2 << 30) > free_b:
+            return {"label": label, "skipped": "needs %.1f GB, %.1f GB free" % (nbytes / 1e9, free_b / 1e9)}
+        arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        cache = B.amskv_cache_create(desc, arena, nbytes)
+        work = algorithmic_work(wl, policies)
+
+        def step(events=None):
+            stream = torch.cuda.current_stream()   # the capture stream while a graph is being recorded
+            B.amskv_cache_reset(cache)
+            for k in range(K):
+                q, kk, v = qkv[k]
+                for layer in range(wl.layers):
+                    B.amskv_append(cache, layer, k, kk, v, stream)
+                    if events is not None:
+                        e0, e1 = events[(layer, k)]
+                        e0.record(stream)
+                        B.amskv_attend(cache, layer, k, q, outs[k], stream)
+                        e1.record(stream)
+                    else:
+                        B.amskv_attend(cache, layer, k, q, outs[k], stream)
+
+        for _ in range(args.warmup):
+            step()
+        torch.cuda.synchronize()
+        assert B.amskv_status(cache) == 0
+        # the launch-bound coarse scales are replayed from a CUDA graph
+        graph = None
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()
+            torch.cuda.synchronize()
+        launches0 = B.amskv_launch_count()
+        step()
+        launches_per_step = B.amskv_launch_count() - launches0
+        torch.cuda.synchronize()
+
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(args.steps):
+            if graph is not None:
+                graph.replay()
+            else:
+                step()
+        t1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = t0.elapsed_time(t1)
+        result = {"label": label, "ms_per_step": ms / args.steps, "launches_per_step": launches_per_step,
+                  "kv_bytes": B.amskv_cache_bytes(cache)[2], "arena_bytes": nbytes}
+
+        if instrument:
+            # per-launch durations of the attention kernel: same steps, eager, CUDA events on the launch stream
+            events = {key: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for key in work}
+            att_ms = {key: 0.0 for key in work}
+            t2, t3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            eager_ms = 0.0
+            for _ in range(args.steps):
+                t2.record(stream)
+                step(events)
+                t3.record(stream)
+                torch.cuda.synchronize()
+                eager_ms += t2.elapsed_time(t3)
+                for key, (e0, e1) in events.items():
+                    att_ms[key] += e0.elapsed_time(e1)
+            result["eager_ms_per_step"] = eager_ms / args.steps
+            result["attend_ms_per_step"] = sum(att_ms.values()) / args.steps
+            result["attend_bytes_per_step"] = sum(b for b, _ in work.values())
+            result["attend_flops_per_step"] = sum(f for _, f in work.values())
+            per_scale = []
+            for k in range(K):
+                b = sum(work[(l, k)][0] for l in range(wl.layers))
+                f = sum(work[(l, k)][1] for l in range(wl.layers))
+                t = sum(att_ms[(l, k)] for l in range(wl.layers)) / args.steps
+                roof = sum(max(work[(l, k)][0] / (hbm_gbs * 1e9), work[(l, k)][1] / (tflops * 1e12))
+                           for l in range(wl.layers)) * 1e3
+                per_scale.append({"scale": k, "tokens": tok[k], "ms": round(t, 4), "gbs": round(b / t / 1e6, 1) if t else None,
+                                  "tflops": round(f / t / 1e9, 1) if t else None, "roofline_ms": round(roof, 4),
+                                  "frac": round(roof / t, 3) if t else None})
+            result["per_scale"] = per_scale
+            result["pass_roofline_ms"] = sum(p["roofline_ms"] for p in per_scale)
+        result["clocks"] = sampler.stop()
+        torch.cuda.synchronize()
+        assert B.amskv_status(cache) == 0
+        result["_cache"] = (cache, arena, desc, keep)
+        return result
+
+    policies = wl.policies(full_retention=args.policy == "full")
+    main = measure(policies, args.policy, instrument=True)
+    if "skipped" in main:
+        raise SystemExit("workload does not fit: " + main["skipped"])
+    cache, arena, desc, keep = main.pop("_cache")
+
+    # end to end through the C ABI with HOST buffers: pinned K/V/Q in, result out, every step
+    e2e = None
+    if not args.no_e2e:
+        nst = B.amskv_step_staging_bytes(cache)
+        staging = torch.empty(nst, dtype=torch.uint8, device="cuda")
+        hq = [q.cpu().pin_memory() for q, _, _ in qkv]
+        hk = [k.cpu().pin_memory() for _, k, _ in qkv]
+        hv = [v.cpu().pin_memory() for _, _, v in qkv]
+        ho = [torch.empty_like(q).pin_memory() for q in hq]
+
+        def host_step():
+            B.amskv_cache_reset(cache)
+            for k in range(K):
+                for layer in range(wl.layers):
+                    B.amskv_step_host(cache, layer, k, hk[k], hv[k], hq[k], ho[k], staging, nst, stream)
+
+        host_step()
+        torch.cuda.synchronize()
+        e_steps = max(1, min(args.steps, args.e2e_steps))
+        if world > 1:
+            dist.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e_steps):
+            host_step()
+        b.record(stream)
+        torch.cuda.synchronize()
+        e_ms = a.elapsed_time(b) / e_steps
+        if world > 1:
+            t = torch.tensor([e_ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = wl.layers * input_bytes
+        d2h = wl.layers * sum(q.numel() * 2 for q in hq)
+        e2e = {"value": e_ms * 1e3 / (wl.batch * world) , "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e_steps, "ms_per_step": e_ms}
+        del staging, hq, hk, hv, ho
+    B.amskv_cache_destroy(cache)
+    del arena
+    torch.cuda.empty_cache()
+
+    # the other policy (full retention when timing AMS-KV and vice versa): KV bytes and latency beside it
+    other = None
+    if not args.no_compare:
+        other_name = "full" if args.policy == "ams" else "ams"
+        other = measure(wl.policies(full_retention=other_name == "full"), other_name, instrument=False)
+        if "_cache" in other:
+            c2, a2, _, _ = other.pop("_cache")
+            B.amskv_cache_destroy(c2)
+            del a2
+            torch.cuda.empty_cache()
+
+    ms = main["ms_per_step"]
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    images = wl.batch * world
+    value = ms * 1e3 / images
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_sample(wl, policies, args.cpu_rows)
+
+    if rank == 0:
+        att_s = main["attend_ms_per_step"] / 1e3
+        achieved = main["attend_bytes_per_step"] / att_s / 1e9
+        traffic = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy))
+        line = {
+            "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms, 4), "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "%s: %d layers, %d heads x %d, batch %d (rows %d), sides %s, condensed %d, local %d, "
+                                   "%d cache-demanding layers, policy %s" % (
+                                       wl.name, wl.layers, wl.heads, wl.head_dim, wl.batch, wl.rows,
+                                       "x".join(map(str, wl.sides)), wl.n_condensed, wl.n_local,
+                                       sum(1 for p in policies if p[2]), args.policy),
+                       "step": "append + attend for every scale and layer",
+                       "l2": "inputs and per-layer KV regions far larger than L2; no flush needed",
+                       "launch": "CUDA graph replay" if not args.no_graph else "eager",
+                       "replicas": world},
+            "clocks": main["clocks"],
+            "e2e": e2e,
+            "gpu_launches": main["launches_per_step"] * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "attention (all attend launches of a step)",
+                         "achieved": round(achieved, 1), "peak": hbm_gbs, "unit": "GB/s",
+                         "frac": round(achieved / hbm_gbs, 4), "peak_kind": peak_kind, "traffic": traffic,
+                         "frac_of_8TBs_nominal": round(achieved / 8000.0, 4)},
+            "pass_roofline": {"roofline_ms": round(main["pass_roofline_ms"], 3),
+                              "attend_ms": round(main["attend_ms_per_step"], 3),
+                              "frac": round(main["pass_roofline_ms"] / main["attend_ms_per_step"], 4),
+                              "note": "sum over launches of max(bytes/HBM peak, flops/bf16 peak) / measured attention time"},
+            "attend_only_us_per_image": round(main["attend_ms_per_step"] * 1e3 / wl.batch, 3),
+            "eager_ms_per_step": round(main["eager_ms_per_step"], 4),
+            "kv_cache_gb": round(main["kv_bytes"] / 1e9, 3),
+            "per_scale": main["per_scale"],
+            "cpu_baseline": cpu_baseline,
+        }
+        if other is not None:
+            if "skipped" in other:
+                line["compare"] = other
+            else:
+                line["compare"] = {"policy": other["label"], "ms_per_step": round(other["ms_per_step"], 4),
+                                   "us_per_image": round(other["ms_per_step"] * 1e3 / wl.batch, 3),
+                                   "kv_cache_gb": round(other["kv_bytes"] / 1e9, 3)}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def oracle_sample(wl, policies, rows):
+    """Times the oracle, as it stands, on a bounded sample of the workload: `rows` rows of one
+    cache-efficient and one cache-demanding layer, all scales.  Work is linear in rows and layers,
+    so the per-image figure for the whole workload is the layer-weighted sum."""
+    import numpy as np
+    import oracle
+    from paper_2511_16047_b200 import synth
+
+    K = len(wl.sides)
+    tok = wl.tokens
+    qkv = [synth.qkv_for_scale(rows, wl.heads, tok[k], wl.head_dim, wl.seed, k, "cpu") for k in range(K)]
+
+    def items(x):
+        return x.double().reshape(rows * wl.heads, x.shape[2], wl.head_dim).numpy()
+
+    Q = [items(q) for q, _, _ in qkv]
+    Ks = [items(k) for _, k, _ in qkv]
+    Vs = [items(v) for _, _, v in qkv]
+    scale = 1.0 / math.sqrt(wl.head_dim)
+    kinds = {}
+    for pol in policies:
+        kinds.setdefault(pol, 0)
+        kinds[pol] += 1
+    total_s = 0.0
+    weighted = 0.0
+    for pol, count in kinds.items():
+        c, w, dem = pol
+        t0 = time.perf_counter()
+        for k in range(K):
+            oracle.attend_selected(Q[k], Ks, Vs, oracle.keep_set(k, c, w, dem), scale)
+        dt = time.perf_counter() - t0
+        total_s += dt
+        weighted += dt * count
+    images = rows / 2.0
+    return {"value": round(weighted * 1e6 / images, 1), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "%d rows x %d heads, one layer of each policy kind (%d kinds), all %d scales: %.1f s measured; "
+                      "value = layer-weighted extrapolation to %d layers" % (rows, wl.heads, len(kinds), K, total_s, wl.layers),
+            "measured_s": round(total_s, 2)}
+
+
+def run_reference(args):
+    """The reference arm: the oracle on the host cores, on the same workload, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2511_16047_b200 import synth
+    wl = synth.WORKLOADS[args.workload]
+    if args.batch:
+        wl = wl.replace(batch=args.batch)
+    policies = wl.policies(full_retention=args.policy == "full")
+    rows = max(2, args.cpu_rows // 4)
+    for _ in range(max(1, min(args.warmup, 1))):
+        oracle_sample(wl, policies, 2)
+    vals, secs = [], 0.0
+    steps = max(1, min(args.steps, 3))
+    for _ in range(steps):
+        r = oracle_sample(wl, policies, rows)
+        vals.append(r["value"])
+        secs += r["measured_s"]
+    value = sum(vals) / len(vals)
+    sample = r["sample"]
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": steps, "warmup": 1, "ms_per_step": round(value * wl.batch / 1e3, 3), "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "policy": args.policy, "note": "fp64 CPU oracle, bounded sample per step"},
+            "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": r["cores"], "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="var_d30")
+    ap.add_argument("--policy", default="ams", choices=["ams", "full"])
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (images)")
+    ap.add_argument("--cpu-rows", type=int, default=64, help="rows of the oracle's timed sample")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-compare", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
