@@ -134,6 +134,8 @@ def run_ours(args):
     wl = synth.WORKLOADS[args.workload]
     if args.batch:
         wl = wl.replace(batch=args.batch)
+    if args.layers:
+        wl = wl.replace(layers=args.layers)
     hbm_gbs, tflops, peak_kind = _peaks()
     K = len(wl.sides)
     tok = wl.tokens
@@ -409,6 +411,8 @@ def run_reference(args):
     wl = synth.WORKLOADS[args.workload]
     if args.batch:
         wl = wl.replace(batch=args.batch)
+    if args.layers:
+        wl = wl.replace(layers=args.layers)
     policies = wl.policies(full_retention=args.policy == "full")
     rows = max(2, args.cpu_rows // 4)
     for _ in range(max(1, min(args.warmup, 1))):
@@ -440,6 +444,7 @@ def main():
     ap.add_argument("--workload", default="var_d30")
     ap.add_argument("--policy", default="ams", choices=["ams", "full"])
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (images)")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
     ap.add_argument("--cpu-rows", type=int, default=64, help="rows of the oracle's timed sample")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-graph", action="store_true")

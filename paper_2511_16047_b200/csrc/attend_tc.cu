@@ -3,15 +3,18 @@
 //
 // Work unit = (row, head, 128-query tile).  A CTA is persistent and walks its units; inside a
 // unit it walks 64-token key/value tiles of the resident ranges.
-//   warp 4      TMA producer: Q tile once per unit, K and V tiles through a 2-stage ring
-//   warp 5      issues tcgen05.mma: S = Q K_j^T (128 x 64, fp32 in TMEM), then O += P_j V_j
+//   warp 4      TMA producer: Q tile per unit (double-buffered for head_dim 64), K and V tiles
+//               through a ring of stages, 16 tokens per bulk copy so a range's tail tile reads
+//               only the 16-token groups it needs
+//   warp 5      issues tcgen05.mma: S_j = Q K_j^T (128 x 64, fp32, two TMEM buffers) one tile
+//               ahead of O += P_j V_j, so the softmax warps always find the next S ready
 //   warps 0-3   one query row per thread (row = TMEM lane): read S with tcgen05.ld, running-max
 //               softmax in exp2 form, write P as bf16 into a swizzled shared tile, and at the end
 //               of the unit read O, divide by the row sum and store bf16 to global memory
 // The accumulator O is rescaled in place only when the row maximum grew by more than 2^8 since
 // the reference maximum was taken, so for well-conditioned logits it is never touched.
-// Each CTA serialises S -> softmax -> PV for one tile; several CTAs per SM overlap each other.
-// Every wait is bounded: a wait that gives up records a status code and the CTA winds down.
+// Two CTAs share an SM.  Every wait is bounded: a wait that gives up records a status code
+// and the CTA winds down.
 #include <cuda.h>  // CUtensorMap and enums only; the encoder is fetched from the driver at run time
 
 #include "kernels.cuh"
@@ -21,34 +24,39 @@ namespace amskv {
 namespace {
 
 constexpr int kQRows = 128;       // query rows per tile = TMEM lanes
+constexpr int kQBoxRows = 32;     // query rows per bulk copy
 constexpr int kKT = 64;           // key/value tokens per tile
-constexpr int kStages = 2;
+constexpr int kKVBoxRows = 16;    // tokens per bulk copy
 constexpr int kThreads = 192;
 constexpr int kProducerWarp = 4;
 constexpr int kMmaWarp = 5;
+constexpr int kMaxStages = 4;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleLog2 = 8.f;
 
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;                      // 128-byte swizzle atoms per row
+    static constexpr int kStages = (D == 64) ? 4 : 2;
+    static constexpr int kQBufs = (D == 64) ? 2 : 1;
     static constexpr uint32_t kQBytes = kQRows * D * 2;
     static constexpr uint32_t kQHalfBytes = kQRows * 128;
     static constexpr uint32_t kKVBytes = kKT * D * 2;           // one K (or V) tile
     static constexpr uint32_t kKVHalfBytes = kKT * 128;
     static constexpr uint32_t kStageBytes = 2 * kKVBytes;
     static constexpr uint32_t kPBytes = kQRows * kKT * 2;
-    static constexpr uint32_t kTileBytes = kQBytes + kStages * kStageBytes + kPBytes;
+    static constexpr uint32_t kTileBytes = kQBufs * kQBytes + kStages * kStageBytes + kPBytes;
     static constexpr uint32_t kSmemBytes = 1024 + kTileBytes;   // barriers + alignment slack in front
-    static constexpr uint32_t kTmemCols = (D == 64) ? 128 : 256;
-    static constexpr uint32_t kSCol = 0, kOCol = kKT;
-    static constexpr int kCtasPerSm = (D == 64) ? 3 : 2;
+    static constexpr uint32_t kTmemCols = 256;                  // S x2 (64 each) + O (D)
+    static constexpr uint32_t kSCol = 0, kOCol = 2 * kKT;
+    static constexpr int kCtasPerSm = 2;
 };
 
 struct Barriers {
-    uint64_t q_full, q_empty;
-    uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_full, p_full, o_full, o_empty;
+    uint64_t q_full[2], q_empty[2];
+    uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
+    uint64_t s_full[2];
+    uint64_t p_full, p_empty, o_full, o_empty;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -147,6 +155,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 64 consecutive fp32 columns of this thread's TMEM lane (two loads, one wait).
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64])
+{
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr), "r"(taddr + 32)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
 {
     asm volatile(
@@ -194,26 +216,18 @@ __device__ __forceinline__ void report(int* status, int code, volatile int* abor
     *abort_flag = 1;
 }
 
-// Walks the 64-token tiles of the resident ranges in order.
-struct TileWalk {
-    const RangeList& rl;
+// Tile j of the resident ranges: first token and number of valid tokens (<= 64).
+__device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0, int32_t& valid)
+{
     int r = 0;
-    int32_t t = 0;
-    __device__ explicit TileWalk(const RangeList& ranges) : rl(ranges) { t = rl.n > 0 ? rl.r[0].start : 0; }
-    __device__ bool next(int32_t& t0, int32_t& valid)
-    {
-        while (r < rl.n && t >= rl.r[r].start + rl.r[r].len) {
-            ++r;
-            if (r < rl.n) t = rl.r[r].start;
-        }
-        if (r >= rl.n) return false;
-        const int32_t end = rl.r[r].start + rl.r[r].len;
-        t0 = t;
-        valid = min(kKT, end - t);
-        t += kKT;
-        return true;
+    for (; r < rl.n - 1; ++r) {
+        const int nt = (rl.r[r].len + kKT - 1) / kKT;
+        if (j < nt) break;
+        j -= nt;
     }
-};
+    t0 = rl.r[r].start + j * kKT;
+    valid = min(kKT, rl.r[r].start + rl.r[r].len - t0);
+}
 
 // ---------------------------------------------------------------- kernel
 template <int D>
@@ -230,22 +244,25 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + (uint32_t)sizeof(Barriers) + 1023u) & ~1023u;
     const uint32_t q_smem = tiles;
-    const uint32_t kv_smem = q_smem + C::kQBytes;
-    const uint32_t p_smem = kv_smem + kStages * C::kStageBytes;
+    const uint32_t kv_smem = q_smem + C::kQBufs * C::kQBytes;
+    const uint32_t p_smem = kv_smem + C::kStages * C::kStageBytes;
     uint8_t* p_generic = smem_raw + (p_smem - raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const bool layout_ok = (tiles + C::kTileBytes) <= (raw + C::kSmemBytes);
     if (threadIdx.x == 0) {
         bars->abort_flag = 0;
-        mbar_init(smem_u32(&bars->q_full), 1);
-        mbar_init(smem_u32(&bars->q_empty), 1);
-        for (int s = 0; s < kStages; ++s) {
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bars->q_full[b]), 1);
+            mbar_init(smem_u32(&bars->q_empty[b]), 1);
+            mbar_init(smem_u32(&bars->s_full[b]), 1);
+        }
+        for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars->kv_full[s]), 1);
             mbar_init(smem_u32(&bars->kv_empty[s]), 1);
         }
-        mbar_init(smem_u32(&bars->s_full), 1);
         mbar_init(smem_u32(&bars->p_full), 4);
+        mbar_init(smem_u32(&bars->p_empty), 1);
         mbar_init(smem_u32(&bars->o_full), 1);
         mbar_init(smem_u32(&bars->o_empty), 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -264,50 +281,67 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
     const uint32_t tmem = bars->tmem_base;
     const uint32_t s_tmem = tmem + C::kSCol, o_tmem = tmem + C::kOCol;
 
-    const uint32_t q_full = smem_u32(&bars->q_full), q_empty = smem_u32(&bars->q_empty);
-    const uint32_t s_full = smem_u32(&bars->s_full), p_full = smem_u32(&bars->p_full);
+    const uint32_t q_full0 = smem_u32(&bars->q_full[0]), q_empty0 = smem_u32(&bars->q_empty[0]);
+    const uint32_t s_full0 = smem_u32(&bars->s_full[0]);
+    const uint32_t p_full = smem_u32(&bars->p_full), p_empty = smem_u32(&bars->p_empty);
     const uint32_t o_full = smem_u32(&bars->o_full), o_empty = smem_u32(&bars->o_empty);
     const uint32_t kv_full0 = smem_u32(&bars->kv_full[0]), kv_empty0 = smem_u32(&bars->kv_empty[0]);
+
+    // units of this CTA: u = blockIdx.x + n * gridDim.x, n = 0 .. my_units-1; every unit has n_tiles tiles
+    const uint32_t my_units = blockIdx.x < n_units ? (uint32_t)((n_units - 1 - blockIdx.x) / gridDim.x + 1) : 0u;
+    const uint32_t total_tiles = my_units * (uint32_t)n_tiles;
 
     if (layout_ok && warp == kProducerWarp) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t n = 0, g = 0;
-            uint32_t armed[kStages] = {0, 0};
+            uint32_t g = 0;
+            uint32_t armed[kMaxStages] = {0, 0, 0, 0};
             bool ok = true;
-            for (int64_t u = blockIdx.x; ok && u < n_units; u += gridDim.x, ++n) {
+            for (uint32_t n = 0; ok && n < my_units; ++n) {
+                const int64_t u = (int64_t)blockIdx.x + (int64_t)n * gridDim.x;
                 const int64_t item = u / nqt;
                 const int32_t qt = (int32_t)(u - item * nqt);
                 const int32_t row = (int32_t)(item / heads), head = (int32_t)(item - (int64_t)row * heads);
-                if (!mbar_wait(q_empty, (n & 1u) ^ 1u, abort_flag)) { report(status, kStatusTmaTimeout, abort_flag); ok = false; break; }
-                mbar_expect_tx(q_full, C::kQBytes);
+                const int32_t valid_rows = min(kQRows, T - qt * kQRows);
+                const uint32_t qb = n % C::kQBufs, quse = n / C::kQBufs;
+                if (!mbar_wait(q_empty0 + 8 * qb, (quse & 1u) ^ 1u, abort_flag)) { report(status, kStatusTmaTimeout, abort_flag); ok = false; break; }
+                const int qboxes = (valid_rows + kQBoxRows - 1) / kQBoxRows;
+                const uint32_t qf = q_full0 + 8 * qb;
+                mbar_expect_tx(qf, (uint32_t)qboxes * kQBoxRows * D * 2);
                 int c[4] = {0, 0, 0, 0};
-                c[qpos.x] = qt * kQRows;
                 c[qpos.y] = head;
                 c[qpos.z] = row;
+                for (int bx = 0; bx < qboxes; ++bx) {
+                    c[qpos.x] = qt * kQRows + bx * kQBoxRows;
 #pragma unroll
-                for (int h = 0; h < C::kHalves; ++h)
-                    tma_load_4d(q_smem + h * C::kQHalfBytes, &q_map, q_full, h * 64, c[1], c[2], c[3]);
-                TileWalk walk(ranges);
-                int32_t t0, valid;
-                while (walk.next(t0, valid)) {
-                    const uint32_t stage = g % kStages, use = g / kStages;
+                    for (int h = 0; h < C::kHalves; ++h)
+                        tma_load_4d(q_smem + qb * C::kQBytes + h * C::kQHalfBytes + bx * kQBoxRows * 128, &q_map, qf,
+                                    h * 64, c[1], c[2], c[3]);
+                }
+                for (int j = 0; j < n_tiles; ++j, ++g) {
+                    int32_t t0, valid;
+                    tile_at(ranges, j, t0, valid);
+                    const uint32_t stage = g % C::kStages, use = g / C::kStages;
                     if (!mbar_wait(kv_empty0 + 8 * stage, (use & 1u) ^ 1u, abort_flag)) { report(status, kStatusTmaTimeout, abort_flag); ok = false; break; }
                     const uint32_t full = kv_full0 + 8 * stage;
-                    mbar_expect_tx(full, C::kStageBytes);
+                    const int nch = (valid + 15) >> 4;
+                    mbar_expect_tx(full, (uint32_t)nch * kKVBoxRows * D * 2 * 2);
                     const uint32_t k_dst = kv_smem + stage * C::kStageBytes, v_dst = k_dst + C::kKVBytes;
+                    for (int bx = 0; bx < nch; ++bx) {
 #pragma unroll
-                    for (int h = 0; h < C::kHalves; ++h) {
-                        tma_load_3d(k_dst + h * C::kKVHalfBytes, &k_map, full, h * 64, t0, (int)item);
-                        tma_load_3d(v_dst + h * C::kKVHalfBytes, &v_map, full, h * 64, t0, (int)item);
+                        for (int h = 0; h < C::kHalves; ++h) {
+                            tma_load_3d(k_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &k_map, full, h * 64,
+                                        t0 + bx * kKVBoxRows, (int)item);
+                            tma_load_3d(v_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &v_map, full, h * 64,
+                                        t0 + bx * kKVBoxRows, (int)item);
+                        }
                     }
                     armed[stage] = use + 1;
-                    ++g;
                 }
             }
             if (!ok) {
                 // wind down: let the copies that were issued land before the CTA gives its shared memory back
-                for (int s = 0; s < kStages; ++s)
+                for (int s = 0; s < C::kStages; ++s)
                     if (armed[s]) {
                         for (uint32_t i = 0; i < kSpinLimit; ++i)
                             if (mbar_try_wait(kv_full0 + 8 * s, (armed[s] - 1) & 1u)) break;
@@ -316,139 +350,146 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
         }
     } else if (layout_ok && warp == kMmaWarp) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            uint32_t n = 0, g = 0;
+        if (lane == 0 && total_tiles > 0) {
             bool ok = true;
             const uint32_t idesc_pv = make_idesc(kQRows, D, 1);
-            for (int64_t u = blockIdx.x; ok && u < n_units; u += gridDim.x, ++n) {
-                TileWalk walk(ranges);
+            // S for flat tile gs: Q of its unit times K of its stage, into S buffer gs % 2
+            auto issue_s = [&](uint32_t gs) -> bool {
+                const uint32_t n = gs / (uint32_t)n_tiles, j = gs - n * (uint32_t)n_tiles;
+                const uint32_t qb = n % C::kQBufs, quse = n / C::kQBufs;
+                const uint32_t stage = gs % C::kStages, use = gs / C::kStages;
                 int32_t t0, valid;
-                int j = 0;
-                while (walk.next(t0, valid)) {
-                    const uint32_t stage = g % kStages, use = g / kStages;
-                    const uint32_t nch = (uint32_t)(valid + 15) >> 4;
-                    const uint32_t k_src = kv_smem + stage * C::kStageBytes, v_src = k_src + C::kKVBytes;
-                    if (!mbar_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) { report(status, kStatusMmaTimeout, abort_flag); ok = false; break; }
-                    if (j == 0 && !mbar_wait(q_full, n & 1u, abort_flag)) { report(status, kStatusMmaTimeout, abort_flag); ok = false; break; }
-                    tc_fence_after();
-                    // S = Q K_j^T : M = 128 queries, N = 16 * nch tokens, K = D channels in steps of 16
-                    const uint32_t idesc_s = make_idesc(kQRows, nch * 16, 0);
+                tile_at(ranges, (int)j, t0, valid);
+                const uint32_t nch = (uint32_t)(valid + 15) >> 4;
+                if (j == 0 && !mbar_wait(q_full0 + 8 * qb, quse & 1u, abort_flag)) return false;
+                if (!mbar_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t q_src = q_smem + qb * C::kQBytes;
+                const uint32_t k_src = kv_smem + stage * C::kStageBytes;
+                const uint32_t idesc_s = make_idesc(kQRows, nch * 16, 0);
+                const uint32_t d = s_tmem + (gs & 1u) * kKT;
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t a = q_smem + (ks >> 2) * C::kQHalfBytes + (ks & 3) * 32;
-                        const uint32_t b = k_src + (ks >> 2) * C::kKVHalfBytes + (ks & 3) * 32;
-                        umma_bf16(s_tmem, make_smem_desc(a, 16, 1024), make_smem_desc(b, 16, 1024), idesc_s, ks > 0);
-                    }
-                    umma_commit(s_full);
-                    if (j == n_tiles - 1) umma_commit(q_empty);
-                    if (!mbar_wait(p_full, g & 1u, abort_flag)) { report(status, kStatusMmaTimeout, abort_flag); ok = false; break; }
-                    if (j == 0 && !mbar_wait(o_empty, (n & 1u) ^ 1u, abort_flag)) { report(status, kStatusMmaTimeout, abort_flag); ok = false; break; }
-                    tc_fence_after();
-                    // O (+)= P_j V_j : M = 128, N = D channels, K = 16 * nch tokens; V is read MN-major
-                    for (uint32_t ks = 0; ks < nch; ++ks) {
-                        const uint64_t a = make_smem_desc(p_smem + ks * 32, 16, 1024);
-                        const uint64_t b = make_smem_desc(v_src + ks * 2048, C::kKVHalfBytes, 1024);
-                        umma_bf16(o_tmem, a, b, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-                    }
-                    umma_commit(kv_empty0 + 8 * stage);
-                    if (j == n_tiles - 1) umma_commit(o_full);
-                    ++j;
-                    ++g;
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t a = q_src + (ks >> 2) * C::kQHalfBytes + (ks & 3) * 32;
+                    const uint32_t b = k_src + (ks >> 2) * C::kKVHalfBytes + (ks & 3) * 32;
+                    umma_bf16(d, make_smem_desc(a, 16, 1024), make_smem_desc(b, 16, 1024), idesc_s, ks > 0);
                 }
+                umma_commit(s_full0 + 8 * (gs & 1u));
+                if (j == (uint32_t)n_tiles - 1) umma_commit(q_empty0 + 8 * qb);
+                return true;
+            };
+            ok = issue_s(0);
+            for (uint32_t g = 0; ok && g < total_tiles; ++g) {
+                // S runs one tile ahead.  Its buffer was last read by the softmax of tile g-1, whose
+                // arrival on p_full was awaited in the previous iteration.
+                if (g + 1 < total_tiles && !issue_s(g + 1)) { ok = false; break; }
+                const uint32_t n = g / (uint32_t)n_tiles, j = g - n * (uint32_t)n_tiles;
+                const uint32_t stage = g % C::kStages;
+                int32_t t0, valid;
+                tile_at(ranges, (int)j, t0, valid);
+                const uint32_t nch = (uint32_t)(valid + 15) >> 4;
+                if (!mbar_wait(p_full, g & 1u, abort_flag)) { ok = false; break; }
+                if (j == 0 && !mbar_wait(o_empty, (n & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                // O (+)= P_j V_j : M = 128, N = D channels, K = 16 * nch tokens; V is read MN-major
+                const uint32_t v_src = kv_smem + stage * C::kStageBytes + C::kKVBytes;
+                for (uint32_t ks = 0; ks < nch; ++ks) {
+                    const uint64_t a = make_smem_desc(p_smem + ks * 32, 16, 1024);
+                    const uint64_t b = make_smem_desc(v_src + ks * 2048, C::kKVHalfBytes, 1024);
+                    umma_bf16(o_tmem, a, b, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                }
+                umma_commit(kv_empty0 + 8 * stage);
+                umma_commit(p_empty);
+                if (j == (uint32_t)n_tiles - 1) umma_commit(o_full);
             }
+            if (!ok) report(status, kStatusMmaTimeout, abort_flag);
         }
     } else if (layout_ok) {
         // ------------------------------------------------------------ softmax + epilogue (warps 0-3)
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
         const int r = warp * 32 + lane;  // query row inside the tile = TMEM lane
-        uint32_t n = 0, g = 0;
+        uint8_t* prow = p_generic + r * 128;
+        uint32_t g = 0;
         bool ok = true;
-        for (int64_t u = blockIdx.x; ok && u < n_units; u += gridDim.x, ++n) {
+        for (uint32_t n = 0; ok && n < my_units; ++n) {
+            const int64_t u = (int64_t)blockIdx.x + (int64_t)n * gridDim.x;
             const int64_t item = u / nqt;
             const int32_t qt = (int32_t)(u - item * nqt);
             const int32_t valid_rows = min(kQRows, T - qt * kQRows);
             const bool warp_live = warp * 32 < valid_rows;
             float m_ref = 0.f, l = 0.f;
-            TileWalk walk(ranges);
-            int32_t t0, valid;
-            int j = 0;
-            while (walk.next(t0, valid)) {
-                if (!mbar_wait(s_full, g & 1u, abort_flag)) { report(status, kStatusSyncTimeout, abort_flag); ok = false; break; }
+            for (int j = 0; j < n_tiles; ++j, ++g) {
+                int32_t t0, valid;
+                tile_at(ranges, j, t0, valid);
+                if (!__all_sync(0xffffffffu, mbar_wait(s_full0 + 8 * (g & 1u), (g >> 1) & 1u, abort_flag))) { report(status, kStatusSyncTimeout, abort_flag); ok = false; break; }
                 tc_fence_after();
                 if (warp_live) {
                     const int nch = (valid + 15) >> 4;
-                    // pass 1: row maximum over the valid columns of this tile
-                    float mt = -INFINITY;
+                    float s[kKT];
+                    tmem_ld64(s_tmem + (g & 1u) * kKT + lane_base, s);
+                    if (valid < kKT) {
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        if (half * 32 < nch * 16) {
-                            float part[32];
-                            tmem_ld32(s_tmem + lane_base + half * 32, part);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (half * 32 + i < valid) mt = fmaxf(mt, part[i]);
-                        }
+                        for (int i = 0; i < kKT; ++i)
+                            if (i >= valid) s[i] = -INFINITY;
                     }
-                    if (j == 0) {
+                    float mt = s[0];
+#pragma unroll
+                    for (int i = 1; i < kKT; ++i) mt = fmaxf(mt, s[i]);
+                    bool grow = false;
+                    if (j == 0) m_ref = mt;
+                    else grow = (mt - m_ref) * scale_log2 > kRescaleLog2;
+                    const bool any_grow = __any_sync(0xffffffffu, grow);
+                    float alpha = 1.f;
+                    if (grow) {
+                        alpha = fast_exp2((m_ref - mt) * scale_log2);
                         m_ref = mt;
-                    } else {
-                        const bool grow = (mt - m_ref) * scale_log2 > kRescaleLog2;
-                        if (__any_sync(0xffffffffu, grow)) {
-                            const float alpha = grow ? fast_exp2((m_ref - mt) * scale_log2) : 1.f;
-#pragma unroll
-                            for (int cblk = 0; cblk < D / 32; ++cblk) {
-                                float o[32];
-                                tmem_ld32(o_tmem + lane_base + cblk * 32, o);
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                                tmem_st32(o_tmem + lane_base + cblk * 32, o);
-                            }
-                            l *= alpha;
-                            if (grow) m_ref = mt;
-                        }
+                        l *= alpha;
                     }
                     const float neg = -m_ref * scale_log2;
+                    uint32_t pk[kKT / 2];
                     float sum = 0.f;
-                    uint8_t* prow = p_generic + r * 128;
-                    // pass 2: probabilities relative to the reference maximum, bf16, into the swizzled P tile
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        if (half * 32 < nch * 16) {
-                            float part[32];
-                            tmem_ld32(s_tmem + lane_base + half * 32, part);
-#pragma unroll
-                            for (int cc = 0; cc < 4; ++cc) {
-                                const int c = half * 4 + cc;
-                                if (c * 8 < nch * 16) {
-                                    uint4 pk;
-                                    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-                                    for (int i = 0; i < 4; ++i) {
-                                        const int col = c * 8 + 2 * i;
-                                        float p0 = fast_exp2(fmaf(part[cc * 8 + 2 * i], scale_log2, neg));
-                                        float p1 = fast_exp2(fmaf(part[cc * 8 + 2 * i + 1], scale_log2, neg));
-                                        if (col >= valid) p0 = 0.f;
-                                        if (col + 1 >= valid) p1 = 0.f;
-                                        sum += p0 + p1;
-                                        h[i] = __floats2bfloat162_rn(p0, p1);
-                                    }
-                                    *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = pk;
-                                }
-                            }
-                        }
+                    for (int i = 0; i < kKT / 2; ++i) {
+                        const float p0 = fast_exp2(fmaf(s[2 * i], scale_log2, neg));
+                        const float p1 = fast_exp2(fmaf(s[2 * i + 1], scale_log2, neg));
+                        sum += p0 + p1;
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                        pk[i] = *reinterpret_cast<const uint32_t*>(&h);
                     }
                     l += sum;
+                    // the previous tile's P V product must be done before P is overwritten or O is rescaled
+                    if (!__all_sync(0xffffffffu, mbar_wait(p_empty, (g & 1u) ^ 1u, abort_flag))) { report(status, kStatusSyncTimeout, abort_flag); ok = false; break; }
+                    if (any_grow) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int cblk = 0; cblk < D / 32; ++cblk) {
+                            float o[32];
+                            tmem_ld32(o_tmem + lane_base + cblk * 32, o);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                            tmem_st32(o_tmem + lane_base + cblk * 32, o);
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < kKT / 8; ++c) {
+                        if (c * 8 < nch * 16)
+                            *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) =
+                                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    }
+                }
+                else {
+                    // A warp without live rows still may not run ahead: its arrival for tile g+1 must not be
+                    // counted in the phase of tile g, so it too waits for the previous P V product.
+                    if (!__all_sync(0xffffffffu, mbar_wait(p_empty, (g & 1u) ^ 1u, abort_flag))) { report(status, kStatusSyncTimeout, abort_flag); ok = false; break; }
                 }
                 tc_fence_before();
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(p_full);
-                ++j;
-                ++g;
             }
             if (!ok) break;
             // epilogue: out = O / l
-            if (!mbar_wait(o_full, n & 1u, abort_flag)) { report(status, kStatusSyncTimeout, abort_flag); ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(o_full, n & 1u, abort_flag))) { report(status, kStatusSyncTimeout, abort_flag); ok = false; break; }
             tc_fence_after();
             if (warp_live) {
                 const float inv = 1.f / l;
@@ -549,7 +590,7 @@ bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, void
     static_assert(sizeof(CUtensorMap) == 128, "tensor map blob size");
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)region.capacity, (cuuint64_t)items};
     const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)region.capacity * D * 2 * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kKT, 1};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kKVBoxRows, 1};
     CUtensorMap km, vm;
     if (!encode_map(&km, region.base, 3, dims, strides, box)) return false;
     if (!encode_map(&vm, region.base + (int64_t)region.capacity * D, 3, dims, strides, box)) return false;
@@ -576,7 +617,7 @@ cudaError_t launch_attend_tc(const Strided& Q, const Strided& O, const LayerRegi
     int pos[3] = {0, 0, 0};
     for (int a = 0; a < 3; ++a) {
         pos[d[a].which] = a + 1;
-        if (d[a].which == 0) box[a + 1] = kQRows;
+        if (d[a].which == 0) box[a + 1] = kQBoxRows;
         if (d[a].stride == 0) strides[a] = 16;  // a broadcast dimension of extent 1
     }
     CUtensorMap qm;

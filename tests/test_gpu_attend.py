@@ -196,3 +196,49 @@ def test_step_host_matches_device_calls():
             B.amskv_step_host(cache.h, 0, k, hk, hv, hq, ho, staging, nbytes)
             torch.cuda.synchronize()
             check_close(ho, want[k], "step_host scale %d" % k)
+
+
+@pytest.mark.parametrize("path", [B.PATH_AUTO, B.PATH_TENSOR], ids=lambda p: PATH_NAMES[p])
+def test_many_units_per_cta_with_partly_idle_query_tiles(path):
+    """More work units than resident CTAs, and query tiles whose upper warps have no rows
+    (169 = 128 + 41 queries), so persistent CTAs walk several units each."""
+    _need(path)
+    sides = (2, 5, 13)
+    rows, heads, D = 10, 70, 64
+    qkv = make_qkv(rows, heads, sides, D, seed=91)
+    with Cache(2, heads, D, rows, sides, [(1, 1, False), (1, 1, True)]) as cache:
+        outs = run_pass(cache, qkv, path)
+        for layer, pol in enumerate(cache.policies):
+            want = oracle_outputs(qkv, pol, 1.0 / math.sqrt(D))
+            for k in range(len(sides)):
+                check_close(outs[layer][k], want[k], "layer %d scale %d" % (layer, k))
+
+
+def test_full_size_rows_sampled_against_oracle():
+    """The VAR-d30 launch shape (512 rows x 30 heads, 680-token schedule) on one cache-efficient and one
+    cache-demanding layer; sampled (row, head) items are compared with the oracle at every scale."""
+    wl = synth.WORKLOADS["var_d30"]
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < 12e9:
+        pytest.skip("needs about 10 GB of device memory")
+    qkv = make_qkv(wl.rows, wl.heads, wl.sides, wl.head_dim, wl.seed)
+    pols = [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)]
+    items = wl.rows * wl.heads
+    g = torch.Generator().manual_seed(7)
+    sample = sorted(set([0, wl.heads - 1, items - wl.heads, items - 1] +
+                        torch.randint(0, items, (60,), generator=g).tolist()))
+    with Cache(2, wl.heads, wl.head_dim, wl.rows, wl.sides, pols) as cache:
+        outs = run_pass(cache, qkv, B.PATH_AUTO)
+        idx = torch.tensor(sample, device="cuda")
+
+        def pick(x):
+            r, h, t, d = x.shape
+            return x.reshape(r * h, t, d)[idx].reshape(len(sample), 1, t, d)
+
+        small = [(pick(q), pick(k), pick(v)) for q, k, v in qkv]
+        for layer, pol in enumerate(pols):
+            want = oracle_outputs(small, pol, 1.0 / math.sqrt(wl.head_dim))
+            for k in range(len(wl.sides)):
+                check_close(pick(outs[layer][k]), want[k], "full-size layer %d scale %d" % (layer, k))
+        # resident KV bytes equal the closed form for these two layers
+        assert B.amskv_cache_bytes(cache.h)[1] == oracle.kv_bytes(wl.sides, pols, wl.rows, wl.heads, wl.head_dim)
