@@ -41,7 +41,7 @@ class AmskvError(RuntimeError):
 
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
-        raise ImportError("libamskv.so is not built: run `python -m paper_2511_16047_b200.build` "
+        raise ImportError("libamskv.so is not built: run `python paper_2511_16047_b200/build.py` "
                           "(there is no fallback implementation)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t

@@ -8,6 +8,22 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _build_native():
+    """The tests load two shared libraries (the CUDA library and the C part of the oracle);
+    both are compiled in-tree here when missing or stale, before anything imports them."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location(
+        "_amskv_build", os.path.join(ROOT, "paper_2511_16047_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build_library()
+    import oracle
+    oracle.build()
+
+
+_build_native()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
