@@ -171,6 +171,30 @@ AMSKV_API int amskv_layer_similarity(const void* K_prev, int side_prev, const vo
 AMSKV_API size_t amskv_similarity_workspace_bytes(void);
 
 /*
+ * amskv_layer_similarity for callers that cannot provide a workspace because they cannot
+ * allocate device memory at the point of the call: code running inside a memory pool whose
+ * budget is fixed, a plug-in that is handed its tensors and nothing else, a real-time or
+ * latency-critical loop in which cudaMalloc (which may synchronise the whole device) is
+ * forbidden.  (The paper has no counterpart of this call; it exists for those callers.)
+ * Same arguments, arithmetic, reduction order and result as amskv_layer_similarity, but the
+ * per-block partial sums go to a 16 KB array that lives inside the library image on every
+ * device that loads it, until the process exits.  The call allocates and frees nothing.
+ *   Limit       rows * heads * side_cur^2 * head_dim / 8 <= 2^30 (16 GiB of current-scale
+ *               keys); larger problems are refused with AMSKV_ERR_UNSUPPORTED, and devices
+ *               with an ordinal of 64 or more likewise.
+ *   First call  on each device looks up the array's device address (with that device
+ *               current); make that first call outside any stream capture.
+ *   Sharing     all calls on a device use the one array.  It keeps whatever the last call
+ *               left there; nothing in it has to start at zero because every slot that is read
+ *               is rewritten by the same call first.  Two calls that overlap on the device (on
+ *               different streams, or from different threads) race on it: serialise them.
+ * Errors: INVALID (null or misaligned pointer, bad side / rows / heads), UNSUPPORTED
+ * (head_dim, size limit, device ordinal), CUDA.
+ */
+AMSKV_API int amskv_layer_similarity_static(const void* K_prev, int side_prev, const void* K_cur, int side_cur,
+                                  int rows, int heads, int head_dim, double* out_ss, void* stream);
+
+/*
  * Layer classification from similarity scores (host-only).
  *   by threshold: demanding[l] = scores[l] < theta (strict; Algorithm 1).
  *   by rank:      the n_demanding lowest-scoring layers are demanding, ties to the lower

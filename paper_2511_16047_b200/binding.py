@@ -59,6 +59,7 @@ def _load() -> ctypes.CDLL:
         "amskv_step_staging_bytes": ([vp, szp], i),
         "amskv_layer_similarity": ([vp, i, vp, i, i, i, i, vp, vp, sz, vp], i),
         "amskv_similarity_workspace_bytes": ([], sz),
+        "amskv_layer_similarity_static": ([vp, i, vp, i, i, i, i, vp, vp], i),
         "amskv_classify_by_threshold": ([dp, i, ctypes.c_double, i32p], i),
         "amskv_classify_lowest": ([dp, i, i, i32p], i),
         "amskv_kept_segments": ([vp, i, i, i32p, i32p], i),
@@ -79,7 +80,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy amskv_cache_reset amskv_append "
            "amskv_attend amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
-           "amskv_similarity_workspace_bytes amskv_classify_by_threshold amskv_classify_lowest "
+           "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
            "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_cache_bytes amskv_status "
            "amskv_launch_count amskv_strerror").split()
 
@@ -187,6 +188,16 @@ def amskv_layer_similarity(K_prev, side_prev: int, K_cur, side_cur: int, rows: i
     _check(lib.amskv_layer_similarity(_addr(K_prev), side_prev, _addr(K_cur), side_cur, rows, heads, head_dim,
                                       _addr(out_ss), _addr(workspace), int(workspace_bytes), _stream(stream)),
            "amskv_layer_similarity")
+
+
+def amskv_layer_similarity_static(K_prev, side_prev: int, K_cur, side_cur: int, rows: int, heads: int, head_dim: int,
+                                  out_ss, stream=None) -> None:
+    """amskv_layer_similarity without a workspace argument, for callers that cannot allocate
+    device memory (fixed memory pools, plug-ins, loops where cudaMalloc is off limits): the
+    partial sums live in a 16 KB array inside the library.  Calls on one device share that
+    array, so they must not overlap on the GPU; problems above 2^30 16-byte chunks are refused."""
+    _check(lib.amskv_layer_similarity_static(_addr(K_prev), side_prev, _addr(K_cur), side_cur, rows, heads, head_dim,
+                                             _addr(out_ss), _stream(stream)), "amskv_layer_similarity_static")
 
 
 def amskv_classify_by_threshold(scores: Sequence[float], theta: float) -> List[bool]:

@@ -5,6 +5,9 @@
 // large, so those reads are served by L1/L2 after the first touch), interpolates in fp32 and
 // accumulates the squared differences.  Blocks reduce in fp64 into a partials array; a second
 // single-block kernel adds the partials in a fixed order, so the result is reproducible.
+#include <mutex>
+
+#include "../../include/amskv.h"
 #include "kernels.cuh"
 
 namespace amskv {
@@ -124,3 +127,71 @@ cudaError_t launch_similarity(const __nv_bfloat16* K_prev, int32_t side_prev, co
 }
 
 }  // namespace amskv
+
+// ---------------------------------------------------------------- entry point without allocation
+//
+// Scratch for the per-block partial sums of amskv_layer_similarity_static, resident in every
+// device that loads this library until the process exits (16 KB).  In host code the name
+// g_static_partials is only a stand-in for the symbol: it is never passed to a kernel.  The
+// device address is looked up once per device with cudaGetSymbolAddress (below) and that
+// pointer is what the kernels get.
+namespace amskv {
+namespace {
+
+static __device__ __align__(256) double g_static_partials[kSimilarityMaxBlocks];
+
+constexpr int kMaxDevices = 64;
+// 16-byte chunks one call may cover: 2^30 chunks = 16 GiB of current-scale keys, which keeps
+// every thread's grid-stride loop at or below 2048 iterations over the fixed 2048 partials.
+constexpr int64_t kStaticMaxChunks = 1ll << 30;
+
+std::mutex g_static_mutex;
+double* g_static_addr[kMaxDevices] = {};
+
+// Device address of g_static_partials on the current device; looked up on first use.
+int static_partials(double** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    if (dev < 0 || dev >= kMaxDevices) return AMSKV_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_partials) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return AMSKV_ERR_CUDA;
+        }
+        g_static_addr[dev] = static_cast<double*>(p);
+    }
+    *out = g_static_addr[dev];
+    return AMSKV_OK;
+}
+
+}  // namespace
+}  // namespace amskv
+
+extern "C" int amskv_layer_similarity_static(const void* K_prev, int side_prev, const void* K_cur, int side_cur,
+                                             int rows, int heads, int head_dim, double* out_ss, void* stream)
+{
+    using namespace amskv;
+    if (!K_prev || !K_cur || !out_ss) return AMSKV_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(K_prev) & 15u) || (reinterpret_cast<uintptr_t>(K_cur) & 15u) ||
+        (reinterpret_cast<uintptr_t>(out_ss) & 7u))
+        return AMSKV_ERR_INVALID;
+    if (side_prev < 1 || side_cur < 1 || side_prev > 4096 || side_cur > 4096 || rows < 1 || heads < 1)
+        return AMSKV_ERR_INVALID;
+    if (head_dim != 64 && head_dim != 128) return AMSKV_ERR_UNSUPPORTED;
+    const int64_t items = (int64_t)rows * heads;
+    const int64_t per_item = (int64_t)side_cur * side_cur * (head_dim / 8);
+    if (items > kStaticMaxChunks / per_item) return AMSKV_ERR_UNSUPPORTED;  // beyond the stated maximum
+    double* partials = nullptr;
+    const int rc = static_partials(&partials);
+    if (rc != AMSKV_OK) return rc;
+    // Every partial the final kernel reads is written by the first kernel of the same call, so
+    // nothing left in the array by an earlier call is ever read and nothing needs clearing.
+    const cudaError_t e = launch_similarity((const __nv_bfloat16*)K_prev, side_prev, (const __nv_bfloat16*)K_cur,
+                                            side_cur, items, head_dim, out_ss, partials,
+                                            static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
+}
