@@ -155,6 +155,8 @@ def run_ours(args):
             return {"label": label, "skipped": "needs %.1f GB, %.1f GB free" % (nbytes / 1e9, free_b / 1e9)}
         arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         cache = B.amskv_cache_create(desc, arena, nbytes)
+        if args.path != "auto":
+            B.amskv_set_attend_path(cache, {"simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR, "pair": B.PATH_TENSOR_PAIR}[args.path])
         work = algorithmic_work(wl, policies)
 
         def step(events=None):
@@ -443,6 +445,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="var_d30")
     ap.add_argument("--policy", default="ams", choices=["ams", "full"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "pair"],
+                    help="force one attention kernel for every scale (default: the library chooses per scale)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (images)")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
     ap.add_argument("--cpu-rows", type=int, default=64, help="rows of the oracle's timed sample")

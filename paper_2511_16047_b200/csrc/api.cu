@@ -38,7 +38,8 @@ struct amskv_cache {
     std::vector<LayerLayout> layout;
     std::vector<size_t> layer_offset;  // bytes from the arena start
     std::vector<int32_t> last_appended;
-    std::vector<TensorMapBlob> k_maps, v_maps;
+    std::vector<TensorMapBlob> k_maps, v_maps;      // 16-token boxes
+    std::vector<TensorMapBlob> k_maps64, v_maps64;  // 64-token boxes (whole tiles)
     bool tc_ready = false;
     char* arena = nullptr;
     size_t arena_bytes = 0;
@@ -191,9 +192,12 @@ int amskv_cache_create(const amskv_desc* desc, void* dev_mem, size_t dev_bytes, 
     if (tc_supported(c->head_dim) && prop.major == 10) {
         c->k_maps.resize(c->layers);
         c->v_maps.resize(c->layers);
+        c->k_maps64.resize(c->layers);
+        c->v_maps64.resize(c->layers);
         bool ok = true;
         for (int l = 0; l < c->layers && ok; ++l)
-            ok = tc_encode_kv_maps(c->region(l), c->items(), c->head_dim, c->k_maps[l].bytes, c->v_maps[l].bytes);
+            ok = tc_encode_kv_maps(c->region(l), c->items(), c->head_dim, 16, c->k_maps[l].bytes, c->v_maps[l].bytes) &&
+                 tc_encode_kv_maps(c->region(l), c->items(), c->head_dim, 64, c->k_maps64[l].bytes, c->v_maps64[l].bytes);
         c->tc_ready = ok;
     }
     *out = c;
@@ -247,8 +251,8 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
 
 int amskv_set_attend_path(amskv_cache* cache, int path)
 {
-    if (!cache || path < AMSKV_PATH_AUTO || path > AMSKV_PATH_TENSOR) return AMSKV_ERR_INVALID;
-    if (path == AMSKV_PATH_TENSOR && !cache->tc_ready) return AMSKV_ERR_UNSUPPORTED;
+    if (!cache || path < AMSKV_PATH_AUTO || path > AMSKV_PATH_TENSOR_PAIR) return AMSKV_ERR_INVALID;
+    if (path >= AMSKV_PATH_TENSOR && !cache->tc_ready) return AMSKV_ERR_UNSUPPORTED;
     cache->path = path;
     return AMSKV_OK;
 }
@@ -271,8 +275,14 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
     for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
     bool tensor = cache->path == AMSKV_PATH_TENSOR ||
                   (cache->path == AMSKV_PATH_AUTO && cache->tc_ready && T > kSmallQueryMaxTokens);
+    const bool pair = cache->path == AMSKV_PATH_TENSOR_PAIR;
     cudaError_t e;
-    if (tensor) {
+    if (pair) {
+        e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes,
+                               cache->k_maps64[layer].bytes, cache->v_maps64[layer].bytes, ranges, T, cache->rows,
+                               cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
+                               cache->sm_count, static_cast<cudaStream_t>(stream));
+    } else if (tensor) {
         e = launch_attend_tc(q, o, cache->region(layer), cache->k_maps[layer].bytes, cache->v_maps[layer].bytes, ranges,
                              T, cache->rows, cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
                              cache->sm_count, static_cast<cudaStream_t>(stream));

@@ -1,0 +1,793 @@
+// Tensor-core attention for sm_100a, paired form: softmax(scale * Q K^T) V over the resident
+// token ranges of one layer, both products on tcgen05 with every accumulator in tensor memory.
+//
+// A CTA is persistent and walks "pairs".  A pair is two streams, A and B, each a (row, head,
+// 128-query tile) that runs through the same number of 64-token key/value tiles:
+//   * more than 128 query tokens: the two streams are two query tiles of ONE item, so each
+//     key/value tile is fetched into shared memory once and used by both;
+//   * at most 128 query tokens: the two streams are two different items with their own tiles.
+// Stream B is absent when the pair has no second member.
+//   warps 0-3    softmax group of stream A: one query row per thread (row = TMEM lane)
+//   warps 4-7    softmax group of stream B
+//   warp 8       TMA producer of the key/value tiles (ring of stages, 16 tokens per bulk copy so a
+//                range's tail tile reads only the 16-token groups it needs)
+//   warp 9       issues tcgen05.mma for both streams, alternating between them
+// Per stream and tile: S = Q K^T (128 x 64 fp32 in TMEM) -> the group reads S with tcgen05.ld,
+// exponentiates in exp2 form against a reference maximum, packs P to bf16 and writes it back
+// over S with tcgen05.st -> O += P V with P read from TMEM.  S and P share their columns, so
+// there is no shared-memory tile for P.  While one group exponentiates, the tensor pipe works
+// for the other.  The reference maximum of a row is the maximum of its first tile; O and the
+// row sum are rescaled only when a later tile exceeds it by more than 2^8, so for
+// well-conditioned logits they are never touched.  The first lane of each group fetches its
+// next query tile as soon as the last S of the current one has landed.
+// Every wait is bounded: a wait that gives up records a status code, all roles wind down,
+// copies in flight are awaited and the tensor memory is freed.
+#include <cuda.h>  // CUtensorMap and enums only; the encoder is fetched from the driver at run time
+
+#include "kernels.cuh"
+
+namespace amskv {
+
+namespace {
+
+constexpr int kQRows = 128;       // query rows per tile = TMEM lanes
+constexpr int kQBoxRows = 32;     // query rows per bulk copy
+constexpr int kKT = 64;           // key/value tokens per tile
+constexpr int kKVBoxRows = 16;    // tokens per bulk copy
+constexpr int kGroupWarps = 4;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kThreads = 320;
+constexpr int kMaxStages = 4;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kRescaleLog2 = 8.f;
+
+template <int D>
+struct Cfg {
+    static constexpr int kHalves = D / 64;                      // 128-byte swizzle atoms per row
+    static constexpr int kStages = 4;
+    static constexpr uint32_t kQBytes = kQRows * D * 2;         // one query tile
+    static constexpr uint32_t kQHalfBytes = kQRows * 128;
+    static constexpr uint32_t kKVBytes = kKT * D * 2;           // one K (or V) tile
+    static constexpr uint32_t kKVHalfBytes = kKT * 128;
+    static constexpr uint32_t kStageBytes = 2 * kKVBytes;
+    static constexpr uint32_t kTileBytes = 2 * kQBytes + kStages * kStageBytes;
+    static constexpr uint32_t kSmemBytes = 4096 + kTileBytes;   // barriers, tile table and alignment slack in front
+    static constexpr uint32_t kTmemCols = (D == 64) ? 256 : 512;  // S x2 (64 each) + O x2 (D each)
+    static constexpr uint32_t kSCol = 0, kOCol = 2 * kKT;
+    static constexpr int kCtasPerSm = (D == 64) ? 2 : 1;
+};
+
+constexpr int kTileTab = 256;     // tiles whose (first token, valid tokens) are tabulated in shared memory
+
+struct Barriers {
+    uint64_t q_full[2];
+    uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
+    uint64_t s_full[2], p_full[2], o_full[2], o_free[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int2 tile_tab[kTileTab];
+};
+
+static_assert(sizeof(Barriers) + 1024 <= 4096, "barrier block must fit in front of the 1024-byte aligned tiles");
+
+// How the pairs of one launch are formed; shared by every role.
+struct PairPlan {
+    int32_t two_q;        // 1: streams are query tiles of one item; 0: streams are two items
+    int32_t nqt;          // query tiles per item
+    int32_t npi;          // pairs per item (two_q) -- else unused
+    int32_t n_items;
+    int32_t n_pairs;
+};
+
+struct Stream {
+    int32_t item;
+    int32_t qt;
+    bool valid;
+};
+
+__device__ __forceinline__ Stream stream_of(const PairPlan& pp, int32_t pair, int g)
+{
+    Stream s;
+    if (pp.two_q) {
+        s.item = pp.npi == 1 ? pair : pair / pp.npi;
+        s.qt = 2 * (pair - s.item * pp.npi) + g;
+        s.valid = s.qt < pp.nqt;
+    } else {
+        s.item = 2 * pair + g;
+        s.qt = 0;
+        s.valid = s.item < pp.n_items;
+    }
+    return s;
+}
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false when it gave up or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred P;\n"
+        "elect.sync _|P, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, P;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
+// Bounded wait by a whole warp; the outcome is the same in every lane.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory matrix descriptors are passed as two 32-bit halves: the low half carries the
+// start address (and the leading offset), the high half is the same for every tile.
+// D (+)= A * B with A and B described in shared memory
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "mov.b64 da, {%1, %3};\n"
+        "mov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
+        : "memory");
+}
+// D (+)= A * B with A in tensor memory (128 lanes x packed 16-bit pairs) and B in shared memory
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                        uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .b64 db;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "mov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+#define AMSKV_R32(r, o)                                                                                               \
+    "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]),   \
+        "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]),            \
+        "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15]), "=r"(r[o + 16]), "=r"(r[o + 17]), "=r"(r[o + 18]),         \
+        "=r"(r[o + 19]), "=r"(r[o + 20]), "=r"(r[o + 21]), "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]),         \
+        "=r"(r[o + 25]), "=r"(r[o + 26]), "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]), "=r"(r[o + 30]),         \
+        "=r"(r[o + 31])
+#define AMSKV_W32(r)                                                                                                  \
+    "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),     \
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),   \
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),   \
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+#define AMSKV_L32                                                                                                     \
+    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                                        \
+    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}"
+#define AMSKV_L32B                                                                                                    \
+    "{%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "                              \
+    "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}"
+
+// 32 consecutive 32-bit columns of this thread's TMEM lane; returns after the data has arrived.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 " AMSKV_L32 ", [%32];\n"
+                 "tcgen05.wait::ld.sync.aligned;\n"
+                 : AMSKV_R32(r, 0)
+                 : "r"(taddr)
+                 : "memory");
+}
+// 64 consecutive columns (two loads, one wait).
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 " AMSKV_L32 ", [%64];\n"
+                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 " AMSKV_L32B ", [%65];\n"
+                 "tcgen05.wait::ld.sync.aligned;\n"
+                 : AMSKV_R32(r, 0), AMSKV_R32(r, 32)
+                 : "r"(taddr), "r"(taddr + 32)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st16_nowait(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 8 columns: load, and store (used by the rare rescale of O, which runs with a full S tile in registers)
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                 "tcgen05.wait::ld.sync.aligned;\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};\n"
+                 "tcgen05.wait::st.sync.aligned;\n"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
+// Shared-memory matrix descriptor for a 128-byte-swizzled tile whose rows are 128 bytes.
+// Low half: start address and leading byte offset, both in 16-byte units.  High half: stride
+// byte offset 1024 (eight 128-byte rows), descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes)
+{
+    return ((addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+// Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, A K-major, B K- or MN-major.
+__device__ __forceinline__ uint32_t make_idesc(uint32_t M, uint32_t N, uint32_t b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ void report(int* status, int code, volatile int* abort_flag)
+{
+    atomicCAS(status, 0, code);
+    *abort_flag = 1;
+}
+
+// Tile j of the resident ranges: first token and number of valid tokens (<= 64).
+__device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0, int32_t& valid)
+{
+    int r = 0;
+    for (; r < rl.n - 1; ++r) {
+        const int nt = (rl.r[r].len + kKT - 1) / kKT;
+        if (j < nt) break;
+        j -= nt;
+    }
+    t0 = rl.r[r].start + j * kKT;
+    valid = min(kKT, rl.r[r].start + rl.r[r].len - t0);
+}
+
+// ---------------------------------------------------------------- kernel
+template <int D>
+__global__ void __launch_bounds__(kThreads, Cfg<D>::kCtasPerSm)
+attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                   const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap k_map64,
+                   const __grid_constant__ CUtensorMap v_map64, __nv_bfloat16* __restrict__ O, int64_t o_row,
+                   int64_t o_head, int64_t o_tok, const RangeList ranges, int32_t T, int32_t heads,
+                   const PairPlan pp, int32_t n_tiles, int3 qpos, float scale_log2, int* __restrict__ status)
+{
+    using C = Cfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_raw);
+    volatile int* abort_flag = &bars->abort_flag;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + (uint32_t)sizeof(Barriers) + 1023u) & ~1023u;
+    const uint32_t q_smem = tiles;
+    const uint32_t kv_smem = q_smem + 2 * C::kQBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const bool layout_ok = (tiles + C::kTileBytes) <= (raw + C::kSmemBytes);
+    if (threadIdx.x == 0) {
+        bars->abort_flag = 0;
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(smem_u32(&bars->q_full[g]), 1);
+            mbar_init(smem_u32(&bars->s_full[g]), 1);
+            mbar_init(smem_u32(&bars->p_full[g]), kGroupWarps);
+            mbar_init(smem_u32(&bars->o_full[g]), 1);
+            mbar_init(smem_u32(&bars->o_free[g]), kGroupWarps);
+        }
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars->kv_full[s]), 1);
+            mbar_init(smem_u32(&bars->kv_empty[s]), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!layout_ok) report(status, kStatusSyncTimeout, abort_flag);
+    }
+    for (int j = threadIdx.x; j < n_tiles && j < kTileTab; j += kThreads) {
+        int32_t t0, valid;
+        tile_at(ranges, j, t0, valid);
+        bars->tile_tab[j] = make_int2(t0, valid);
+    }
+    if (layout_ok) {
+        // query rows a tile does not cover keep whatever the slot held before; start them at zero
+        uint4* qz = reinterpret_cast<uint4*>(smem_raw + (q_smem - raw));
+        for (uint32_t i = threadIdx.x; i < 2 * C::kQBytes / 16; i += kThreads) qz[i] = make_uint4(0, 0, 0, 0);
+        fence_async_smem();
+    }
+    if (warp == kProducerWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)),
+                     "r"(C::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    auto tile_of = [&](int j, int32_t& t0, int32_t& valid) {
+        if (j < kTileTab) {
+            const int2 e = bars->tile_tab[j];
+            t0 = e.x;
+            valid = e.y;
+        } else {
+            tile_at(ranges, j, t0, valid);
+        }
+    };
+
+    const uint32_t q_full0 = smem_u32(&bars->q_full[0]);
+    const uint32_t s_full0 = smem_u32(&bars->s_full[0]), p_full0 = smem_u32(&bars->p_full[0]);
+    const uint32_t o_full0 = smem_u32(&bars->o_full[0]), o_free0 = smem_u32(&bars->o_free[0]);
+    const uint32_t kv_full0 = smem_u32(&bars->kv_full[0]), kv_empty0 = smem_u32(&bars->kv_empty[0]);
+
+    // pairs of this CTA: p = blockIdx.x + n * gridDim.x, n = 0 .. my_pairs-1
+    const uint32_t my_pairs = (int32_t)blockIdx.x < pp.n_pairs ? ((uint32_t)pp.n_pairs - 1u - blockIdx.x) / gridDim.x + 1u : 0u;
+
+    // The producer and the MMA issuer run their loops with the whole warp converged and let one
+    // elected lane issue: addresses, descriptors and coordinates then stay warp-uniform values,
+    // which keeps the per-instruction issue cost of the TMA and tcgen05 instructions low.
+    if (layout_ok && warp == kProducerWarp) {
+        // ------------------------------------------------------------ TMA producer of K/V tiles
+        uint32_t sq = 0;  // stages issued so far
+        bool ok = true;
+        for (uint32_t n = 0; ok && n < my_pairs; ++n) {
+            const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
+            const Stream sa = stream_of(pp, pair, 0), sb = stream_of(pp, pair, 1);
+            const int per_tile = (!pp.two_q && sb.valid) ? 2 : 1;
+            for (int j = 0; ok && j < n_tiles; ++j) {
+                int32_t t0, valid;
+                tile_of(j, t0, valid);
+                const int nch = (valid + 15) >> 4;
+                for (int g = 0; g < per_tile; ++g, ++sq) {
+                    const int item = g == 0 ? sa.item : sb.item;
+                    const uint32_t stage = sq % C::kStages, use = sq / C::kStages;
+                    if (!warp_wait(kv_empty0 + 8 * stage, (use & 1u) ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t full = kv_full0 + 8 * stage;
+                    const uint32_t k_dst = kv_smem + stage * C::kStageBytes, v_dst = k_dst + C::kKVBytes;
+                    if (elect_one()) {
+                        mbar_expect_tx(full, (uint32_t)nch * kKVBoxRows * D * 2 * 2);
+                        if (nch == kKT / kKVBoxRows) {
+#pragma unroll
+                            for (int h = 0; h < C::kHalves; ++h) {
+                                tma_load_3d(k_dst + h * C::kKVHalfBytes, &k_map64, full, h * 64, t0, item);
+                                tma_load_3d(v_dst + h * C::kKVHalfBytes, &v_map64, full, h * 64, t0, item);
+                            }
+                        } else {
+                            for (int bx = 0; bx < nch; ++bx) {
+#pragma unroll
+                                for (int h = 0; h < C::kHalves; ++h) {
+                                    tma_load_3d(k_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &k_map, full, h * 64,
+                                                t0 + bx * kKVBoxRows, item);
+                                    tma_load_3d(v_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &v_map, full, h * 64,
+                                                t0 + bx * kKVBoxRows, item);
+                                }
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (!ok) {
+            if (lane == 0) report(status, kStatusTmaTimeout, abort_flag);
+            // wind down: let the copies that were issued land before the CTA gives its shared memory back
+            const uint32_t first = sq > (uint32_t)C::kStages ? sq - C::kStages : 0u;
+            for (uint32_t q = first; q < sq; ++q) {
+                const uint32_t stage = q % C::kStages, use = q / C::kStages;
+                for (uint32_t i = 0; i < kSpinLimit; ++i)
+                    if (mbar_try_wait(kv_full0 + 8 * stage, use & 1u)) break;
+            }
+        }
+    } else if (layout_ok && warp == kMmaWarp) {
+        // ------------------------------------------------------------ MMA issuer
+        if (my_pairs > 0) {
+            bool ok = true;
+            const uint32_t idesc_pv = make_idesc(kQRows, D, 1);
+            const uint32_t k_lo0 = desc_lo(kv_smem, 16);                             // K tile of stage 0, K-major
+            const uint32_t v_lo0 = desc_lo(kv_smem + C::kKVBytes, C::kKVHalfBytes);  // V tile of stage 0, MN-major
+            const uint32_t q_lo0 = desc_lo(q_smem, 16);
+            constexpr uint32_t kStageLo = C::kStageBytes >> 4, kQLo = C::kQBytes >> 4;
+            // per stream: the tile whose S was issued last and whose P V is still to be issued
+            uint32_t pv_stage[2] = {0, 0}, pv_nch[2] = {0, 0};
+            bool pv_live[2] = {false, false}, pv_first[2] = {false, false}, pv_release[2] = {false, false},
+                 pv_last[2] = {false, false};
+            uint32_t tcount[2] = {0, 0};   // tiles issued per stream
+            uint32_t ucount[2] = {0, 0};   // units started per stream
+            uint32_t sq = 0;
+
+            // O (+)= P V : M = 128, N = D channels, K = 16 * nch tokens; P from TMEM (packed over S),
+            // V read MN-major from its stage
+            auto issue_pv = [&](const int g) -> bool {
+                const uint32_t t = tcount[g] - 1;  // flat tile index of this stream
+                if (!warp_wait(p_full0 + 8 * g, t & 1u, abort_flag)) return false;
+                if (pv_first[g] && !warp_wait(o_free0 + 8 * g, ((ucount[g] - 1) & 1u) ^ 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t v_lo = v_lo0 + pv_stage[g] * kStageLo;
+                const uint32_t p_tmem = tmem + C::kSCol + g * kKT;
+                const uint32_t o_tmem = tmem + C::kOCol + g * D;
+                const uint32_t nch = pv_nch[g];
+                if (elect_one()) {
+                    umma_ts(o_tmem, p_tmem, v_lo, kDescHi, idesc_pv, pv_first[g] ? 0u : 1u);
+                    if (nch > 1) umma_ts(o_tmem, p_tmem + 8, v_lo + (2048 >> 4), kDescHi, idesc_pv, 1u);
+                    if (nch > 2) umma_ts(o_tmem, p_tmem + 16, v_lo + (4096 >> 4), kDescHi, idesc_pv, 1u);
+                    if (nch > 3) umma_ts(o_tmem, p_tmem + 24, v_lo + (6144 >> 4), kDescHi, idesc_pv, 1u);
+                    if (pv_release[g]) umma_commit(kv_empty0 + 8 * pv_stage[g]);
+                    if (pv_last[g]) umma_commit(o_full0 + 8 * g);
+                }
+                __syncwarp();
+                return true;
+            };
+
+            for (uint32_t n = 0; ok && n < my_pairs; ++n) {
+                const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
+                const int ng = stream_of(pp, pair, 1).valid ? 2 : 1;
+                for (int j = 0; ok && j < n_tiles; ++j) {
+                    int32_t t0, valid;
+                    tile_of(j, t0, valid);
+                    const uint32_t nch = (uint32_t)(valid + 15) >> 4;
+                    const uint32_t idesc_s = make_idesc(kQRows, nch * 16, 0);
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        if (!ok || g >= ng) continue;
+                        if (pv_live[g] && !issue_pv(g)) { ok = false; continue; }
+                        // S = Q K^T for (stream g, tile j)
+                        const uint32_t seq = pp.two_q ? sq : sq + g;
+                        const uint32_t stage = seq % C::kStages, use = seq / C::kStages;
+                        if (j == 0) {
+                            if (!warp_wait(q_full0 + 8 * g, ucount[g] & 1u, abort_flag)) { ok = false; continue; }
+                            ++ucount[g];
+                        }
+                        if (!(pp.two_q && g == 1)) {  // the second stream of a shared tile finds it landed already
+                            if (!warp_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) { ok = false; continue; }
+                        }
+                        tc_fence_after();
+                        const uint32_t q_lo = q_lo0 + g * kQLo;
+                        const uint32_t k_lo = k_lo0 + stage * kStageLo;
+                        const uint32_t d = tmem + C::kSCol + g * kKT;
+                        if (elect_one()) {
+                            umma_ss<false>(d, q_lo, k_lo, kDescHi, idesc_s);
+#pragma unroll
+                            for (int ks = 1; ks < D / 16; ++ks) {
+                                constexpr uint32_t kQH = C::kQHalfBytes >> 4, kKH = C::kKVHalfBytes >> 4;
+                                umma_ss<true>(d, q_lo + (ks >> 2) * kQH + (ks & 3) * 2,
+                                              k_lo + (ks >> 2) * kKH + (ks & 3) * 2, kDescHi, idesc_s);
+                            }
+                            umma_commit(s_full0 + 8 * g);
+                        }
+                        __syncwarp();
+                        pv_live[g] = true;
+                        pv_stage[g] = stage;
+                        pv_nch[g] = nch;
+                        pv_first[g] = (j == 0);
+                        pv_last[g] = (j == n_tiles - 1);
+                        pv_release[g] = pp.two_q ? (g == ng - 1) : true;
+                        ++tcount[g];
+                    }
+                    sq += pp.two_q ? 1 : ng;
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+                if (ok && pv_live[g] && !issue_pv(g)) ok = false;
+            if (!ok && lane == 0) report(status, kStatusMmaTimeout, abort_flag);
+        }
+    } else if (layout_ok) {
+        // ------------------------------------------------------------ softmax + epilogue (warps 0-7)
+        const int g = warp >> 2, wq = warp & 3;
+        const uint32_t lane_base = ((uint32_t)(wq * 32)) << 16;
+        const int r = wq * 32 + lane;  // query row inside the tile = TMEM lane
+        const uint32_t s_tmem = tmem + C::kSCol + g * kKT + lane_base;
+        const uint32_t o_tmem = tmem + C::kOCol + g * D + lane_base;
+        const uint32_t q_full = q_full0 + 8 * g, s_full = s_full0 + 8 * g, p_full = p_full0 + 8 * g;
+        const uint32_t o_full = o_full0 + 8 * g, o_free = o_free0 + 8 * g;
+        const bool q_loader = (wq == 0 && lane == 0);
+        uint32_t q_armed = 0;
+
+        // fetch the query tile of the first unit at or after pair index n (first lane of the group only)
+        auto load_q = [&](uint32_t n_from) {
+            for (uint32_t n = n_from; n < my_pairs; ++n) {
+                const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
+                const Stream s = stream_of(pp, pair, g);
+                if (!s.valid) continue;
+                const int32_t row = s.item / heads, head = s.item - row * heads;
+                const int32_t valid_rows = min(kQRows, T - s.qt * kQRows);
+                const int qboxes = (valid_rows + kQBoxRows - 1) / kQBoxRows;
+                mbar_expect_tx(q_full, (uint32_t)qboxes * kQBoxRows * D * 2);
+                int c[4] = {0, 0, 0, 0};
+                c[qpos.y] = head;
+                c[qpos.z] = row;
+                for (int bx = 0; bx < qboxes; ++bx) {
+                    c[qpos.x] = s.qt * kQRows + bx * kQBoxRows;
+#pragma unroll
+                    for (int h = 0; h < C::kHalves; ++h)
+                        tma_load_4d(q_smem + g * C::kQBytes + h * C::kQHalfBytes + bx * kQBoxRows * 128, &q_map, q_full,
+                                    h * 64, c[1], c[2], c[3]);
+                }
+                ++q_armed;
+                return;
+            }
+        };
+        if (q_loader) load_q(0);
+
+        uint32_t t = 0;   // flat tile counter of this stream
+        uint32_t un = 0;  // units done by this stream
+        bool ok = true;
+        for (uint32_t n = 0; ok && n < my_pairs; ++n) {
+            const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
+            const Stream st = stream_of(pp, pair, g);
+            if (!st.valid) continue;
+            const int32_t valid_rows = min(kQRows, T - st.qt * kQRows);
+            const bool warp_live = wq * 32 < valid_rows;
+            float m_ref = 0.f, nb = 0.f, l = 0.f;
+            for (int j = 0; j < n_tiles; ++j, ++t) {
+                int32_t t0, valid;
+                tile_of(j, t0, valid);
+                if (!__all_sync(0xffffffffu, mbar_wait(s_full, t & 1u, abort_flag))) {
+                    report(status, kStatusSyncTimeout, abort_flag);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                // the last S of this unit has landed, so its query tile is no longer read
+                if (j == n_tiles - 1 && q_loader) load_q(n + 1);
+                if (warp_live) {
+                    uint32_t sr[kKT];
+                    tmem_ld64(s_tmem, sr);
+                    if (valid < kKT) {
+#pragma unroll
+                        for (int i = 0; i < kKT; ++i)
+                            if (i >= valid) sr[i] = 0xff800000u;  // -inf
+                    }
+                    // row maximum with four independent chains
+                    float mx[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        mx[c] = max3(__uint_as_float(sr[c]), __uint_as_float(sr[4 + c]), __uint_as_float(sr[8 + c]));
+#pragma unroll
+                    for (int i = 12; i < kKT - 4; i += 8) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            mx[c] = max3(mx[c], __uint_as_float(sr[i + c]), __uint_as_float(sr[i + 4 + c]));
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(sr[kKT - 4 + c]));
+                    const float mt = fmaxf(max3(mx[0], mx[1], mx[2]), mx[3]);
+                    if (j == 0) {
+                        m_ref = mt;
+                        nb = -mt * scale_log2;
+                    } else {
+                        const bool grow = fmaf(mt, scale_log2, nb) > kRescaleLog2;
+                        if (__any_sync(0xffffffffu, grow)) {
+                            // rare: bring O and the row sum to the new reference.  The previous P V is done:
+                            // it was issued before this tile's S, whose arrival covers every earlier product.
+                            float alpha = 1.f;
+                            if (grow) {
+                                alpha = fast_exp2((m_ref - mt) * scale_log2);
+                                m_ref = mt;
+                                nb = -mt * scale_log2;
+                                l *= alpha;
+                            }
+#pragma unroll 1
+                            for (int cblk = 0; cblk < D / 8; ++cblk) {
+                                uint32_t o[8];
+                                tmem_ld8(o_tmem + cblk * 8, o);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                tmem_st8(o_tmem + cblk * 8, o);
+                            }
+                        }
+                    }
+                    // P over S: columns 0..31 receive the 64 probabilities as bf16 pairs, 32 tokens per store
+                    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t pk[kKT / 4];
+#pragma unroll
+                        for (int i = 0; i < kKT / 4; ++i) {
+                            const int c = half * (kKT / 2) + 2 * i;
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), scale_log2, nb));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), scale_log2, nb));
+                            sum0 += p0;
+                            sum1 += p1;
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                            pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        tmem_st16_nowait(s_tmem + half * (kKT / 4), pk);
+                    }
+                    l += sum0 + sum1;
+                    tmem_wait_st();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full);
+            }
+            if (!ok) break;
+            // epilogue: out = O / l once the last P V of the unit is done
+            if (!__all_sync(0xffffffffu, mbar_wait(o_full, un & 1u, abort_flag))) {
+                report(status, kStatusSyncTimeout, abort_flag);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            if (warp_live) {
+                const float inv = 1.f / l;
+                const int32_t row = st.item / heads, head = st.item - row * heads;
+                __nv_bfloat16* dst = O + row * o_row + head * o_head + (int64_t)(st.qt * kQRows + r) * o_tok;
+#pragma unroll
+                for (int cblk = 0; cblk < D / 32; ++cblk) {
+                    uint32_t o[32];
+                    tmem_ld32(o_tmem + cblk * 32, o);
+                    if (r < valid_rows) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint4 out4;
+                            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&out4);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                h[i] = __floats2bfloat162_rn(__uint_as_float(o[c * 8 + 2 * i]) * inv,
+                                                             __uint_as_float(o[c * 8 + 2 * i + 1]) * inv);
+                            reinterpret_cast<uint4*>(dst + cblk * 32)[c] = out4;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(o_free);
+            ++un;
+        }
+        // wind down: a query tile requested but never consumed must land before the CTA exits
+        if (q_loader && q_armed > un) {
+            for (uint32_t i = 0; i < kSpinLimit; ++i)
+                if (mbar_try_wait(q_full, (q_armed - 1) & 1u)) break;
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kProducerWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+template <int D>
+cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& km64,
+                   const CUtensorMap& vm64, const Strided& O,
+                   const RangeList& ranges, int32_t T, int32_t heads, const PairPlan& pp, int32_t n_tiles, int3 qpos,
+                   float scale_log2, int* status, int sm_count, cudaStream_t stream)
+{
+    using C = Cfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attend_pair_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
+    if (grid > pp.n_pairs) grid = pp.n_pairs;
+    attend_pair_kernel<D><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(
+        qm, km, vm, km64, vm64, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos, scale_log2,
+        status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map, const void* v_map,
+                               const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
+                               float softmax_scale, int* status, int sm_count, cudaStream_t stream)
+{
+    if (ranges.n < 1 || ranges.total < 1 || T < 1) return cudaErrorInvalidValue;
+    CUtensorMap qm;
+    int pos[3];
+    if (!tc_encode_q_map(Q, T, rows, heads, D, kQBoxRows, &qm, pos)) return cudaErrorNotSupported;
+    CUtensorMap km, vm, km64, vm64;
+    memcpy(&km, k_map, sizeof(km));
+    memcpy(&vm, v_map, sizeof(vm));
+    memcpy(&km64, k_map64, sizeof(km64));
+    memcpy(&vm64, v_map64, sizeof(vm64));
+    PairPlan pp;
+    pp.nqt = (T + kQRows - 1) / kQRows;
+    pp.two_q = pp.nqt >= 2 ? 1 : 0;
+    pp.npi = (pp.nqt + 1) / 2;
+    if ((int64_t)rows * heads > 0x3fffffffll) return cudaErrorInvalidValue;
+    pp.n_items = rows * heads;
+    pp.n_pairs = pp.two_q ? pp.n_items * pp.npi : (pp.n_items + 1) / 2;
+    int32_t n_tiles = 0;
+    for (int i = 0; i < ranges.n; ++i) n_tiles += (ranges.r[i].len + kKT - 1) / kKT;
+    const int3 qpos = make_int3(pos[0], pos[1], pos[2]);
+    const float scale_log2 = softmax_scale * 1.4426950408889634f;
+    if (D == 64)
+        return launch<64>(qm, km, vm, km64, vm64, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status, sm_count, stream);
+    return launch<128>(qm, km, vm, km64, vm64, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status, sm_count, stream);
+}
+
+}  // namespace amskv

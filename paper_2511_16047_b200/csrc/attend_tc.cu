@@ -585,17 +585,42 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
 
 bool tc_supported(int32_t D) { return D == 64 || D == 128; }
 
-bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, void* k_map_out, void* v_map_out)
+bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, int box_rows, void* k_map_out,
+                       void* v_map_out)
 {
     static_assert(sizeof(CUtensorMap) == 128, "tensor map blob size");
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)region.capacity, (cuuint64_t)items};
     const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)region.capacity * D * 2 * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kKVBoxRows, 1};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     CUtensorMap km, vm;
     if (!encode_map(&km, region.base, 3, dims, strides, box)) return false;
     if (!encode_map(&vm, region.base + (int64_t)region.capacity * D, 3, dims, strides, box)) return false;
     memcpy(k_map_out, &km, sizeof(km));
     memcpy(v_map_out, &vm, sizeof(vm));
+    return true;
+}
+
+// Q as a rank-4 tensor: channels, then token / head / row ordered by ascending stride.  pos[0..2]
+// receive the coordinate index (1..3) of the token, head and row dimensions.
+bool tc_encode_q_map(const Strided& Q, int32_t T, int32_t rows, int32_t heads, int32_t D, int box_rows, void* map_out,
+                     int pos[3])
+{
+    struct Dim { cuuint64_t size; int64_t stride; int which; };
+    Dim d[3] = {{(cuuint64_t)T, Q.token, 0}, {(cuuint64_t)heads, Q.head, 1}, {(cuuint64_t)rows, Q.row, 2}};
+    for (int a = 0; a < 3; ++a)
+        for (int b = a + 1; b < 3; ++b)
+            if (d[b].stride < d[a].stride) { Dim t = d[a]; d[a] = d[b]; d[b] = t; }
+    cuuint64_t dims[4] = {(cuuint64_t)D, d[0].size, d[1].size, d[2].size};
+    cuuint64_t strides[3] = {(cuuint64_t)d[0].stride * 2, (cuuint64_t)d[1].stride * 2, (cuuint64_t)d[2].stride * 2};
+    cuuint32_t box[4] = {64, 1, 1, 1};
+    for (int a = 0; a < 3; ++a) {
+        pos[d[a].which] = a + 1;
+        if (d[a].which == 0) box[a + 1] = (cuuint32_t)box_rows;
+        if (d[a].stride == 0) strides[a] = 16;  // a broadcast dimension of extent 1
+    }
+    CUtensorMap qm;
+    if (!encode_map(&qm, Q.ptr, 4, dims, strides, box)) return false;
+    memcpy(map_out, &qm, sizeof(qm));
     return true;
 }
 
@@ -605,23 +630,9 @@ cudaError_t launch_attend_tc(const Strided& Q, const Strided& O, const LayerRegi
 {
     (void)region;
     if (ranges.n < 1 || ranges.total < 1 || T < 1) return cudaErrorInvalidValue;
-    // Q as a rank-4 tensor (D, then token / head / row ordered by ascending stride)
-    struct Dim { cuuint64_t size; int64_t stride; int which; };
-    Dim d[3] = {{(cuuint64_t)T, Q.token, 0}, {(cuuint64_t)heads, Q.head, 1}, {(cuuint64_t)rows, Q.row, 2}};
-    for (int a = 0; a < 3; ++a)
-        for (int b = a + 1; b < 3; ++b)
-            if (d[b].stride < d[a].stride) { Dim t = d[a]; d[a] = d[b]; d[b] = t; }
-    cuuint64_t dims[4] = {(cuuint64_t)D, d[0].size, d[1].size, d[2].size};
-    cuuint64_t strides[3] = {(cuuint64_t)d[0].stride * 2, (cuuint64_t)d[1].stride * 2, (cuuint64_t)d[2].stride * 2};
-    cuuint32_t box[4] = {64, 1, 1, 1};
-    int pos[3] = {0, 0, 0};
-    for (int a = 0; a < 3; ++a) {
-        pos[d[a].which] = a + 1;
-        if (d[a].which == 0) box[a + 1] = kQBoxRows;
-        if (d[a].stride == 0) strides[a] = 16;  // a broadcast dimension of extent 1
-    }
     CUtensorMap qm;
-    if (!encode_map(&qm, Q.ptr, 4, dims, strides, box)) return cudaErrorNotSupported;
+    int pos[3];
+    if (!tc_encode_q_map(Q, T, rows, heads, D, kQBoxRows, &qm, pos)) return cudaErrorNotSupported;
     CUtensorMap km, vm;
     memcpy(&km, k_map, sizeof(km));
     memcpy(&vm, v_map, sizeof(vm));

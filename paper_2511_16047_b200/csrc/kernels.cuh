@@ -57,10 +57,20 @@ cudaError_t launch_similarity(const __nv_bfloat16* K_prev, int32_t side_prev, co
 struct TcMaps;  // defined in attend_tc.cu
 bool tc_supported(int32_t D);
 // Encodes the tensor maps a layer needs for its K and V streams; returns false on failure.
-bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, void* k_map_out, void* v_map_out);
+// (box = 64 channels x box_rows tokens of one item)
+bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, int box_rows, void* k_map_out,
+                       void* v_map_out);
 cudaError_t launch_attend_tc(const Strided& Q, const Strided& O, const LayerRegion& region, const void* k_map,
                              const void* v_map, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads,
                              int32_t D, float softmax_scale, int* status, int sm_count, cudaStream_t stream);
+
+// Encodes the rank-4 tensor map of a strided Q tensor (box = 64 channels x box_rows tokens).
+bool tc_encode_q_map(const Strided& Q, int32_t T, int32_t rows, int32_t heads, int32_t D, int box_rows, void* map_out,
+                     int pos[3]);
+// Paired tensor-core kernel: two softmax groups per CTA, probabilities kept in tensor memory.
+cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map16, const void* v_map16,
+                               const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
+                               float softmax_scale, int* status, int sm_count, cudaStream_t stream);
 
 void count_launch(int n = 1);
 

@@ -13,12 +13,12 @@ from gpu_common import (Cache, check_close, make_qkv, oracle_outputs, run_pass, 
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [B.PATH_SIMT, B.PATH_AUTO, B.PATH_TENSOR]
-PATH_NAMES = {B.PATH_SIMT: "simt", B.PATH_AUTO: "auto", B.PATH_TENSOR: "tensor"}
+PATHS = [B.PATH_SIMT, B.PATH_AUTO, B.PATH_TENSOR, B.PATH_TENSOR_PAIR]
+PATH_NAMES = {B.PATH_SIMT: "simt", B.PATH_AUTO: "auto", B.PATH_TENSOR: "tensor", B.PATH_TENSOR_PAIR: "pair"}
 
 
 def _need(path, head_dim=64):
-    if path == B.PATH_TENSOR and not tensor_path_available(head_dim):
+    if path in (B.PATH_TENSOR, B.PATH_TENSOR_PAIR) and not tensor_path_available(head_dim):
         pytest.skip("tensor-core path not available for head_dim %d" % head_dim)
 
 
@@ -198,7 +198,7 @@ def test_step_host_matches_device_calls():
             check_close(ho, want[k], "step_host scale %d" % k)
 
 
-@pytest.mark.parametrize("path", [B.PATH_AUTO, B.PATH_TENSOR], ids=lambda p: PATH_NAMES[p])
+@pytest.mark.parametrize("path", [B.PATH_AUTO, B.PATH_TENSOR, B.PATH_TENSOR_PAIR], ids=lambda p: PATH_NAMES[p])
 def test_many_units_per_cta_with_partly_idle_query_tiles(path):
     """More work units than resident CTAs, and query tiles whose upper warps have no rows
     (169 = 128 + 41 queries), so persistent CTAs walk several units each."""
