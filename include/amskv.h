@@ -56,9 +56,9 @@ extern "C" {
                                    For sizing and for inspecting the policy without a GPU. */
 
 /* amskv_set_attend_path */
-#define AMSKV_PATH_AUTO 0   /* small-query kernel for few query tokens, tensor cores otherwise */
+#define AMSKV_PATH_AUTO 0   /* small-query kernel for 1-4 query tokens, paired tcgen05 kernel otherwise */
 #define AMSKV_PATH_SIMT 1   /* always the CUDA-core kernel                                     */
-#define AMSKV_PATH_TENSOR 2 /* always the tcgen05 kernel                                       */
+#define AMSKV_PATH_TENSOR 2 /* always the single-stream tcgen05 kernel                         */
 #define AMSKV_PATH_TENSOR_PAIR 3 /* always the paired tcgen05 kernel (two query tiles per CTA)  */
 
 typedef struct amskv_cache amskv_cache; /* opaque; owned by the library */

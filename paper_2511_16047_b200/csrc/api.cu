@@ -16,7 +16,7 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 constexpr size_t kAlign = 256;
 constexpr size_t kStatusBytes = 256;
-constexpr int kSmallQueryMaxTokens = 16;  // scales with at most this many query tokens use the CUDA-core kernel
+constexpr int kSmallQueryMaxTokens = 4;  // scales with at most this many query tokens use the CUDA-core kernel (measured crossover)
 
 static size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -273,9 +273,9 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
     ranges.n = cache->layout[layer].ranges(cache->tokens, scale, ranges.r);
     ranges.total = 0;
     for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
-    bool tensor = cache->path == AMSKV_PATH_TENSOR ||
-                  (cache->path == AMSKV_PATH_AUTO && cache->tc_ready && T > kSmallQueryMaxTokens);
-    const bool pair = cache->path == AMSKV_PATH_TENSOR_PAIR;
+    const bool tensor = cache->path == AMSKV_PATH_TENSOR;
+    const bool pair = cache->path == AMSKV_PATH_TENSOR_PAIR ||
+                      (cache->path == AMSKV_PATH_AUTO && cache->tc_ready && T > kSmallQueryMaxTokens);
     cudaError_t e;
     if (pair) {
         e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes,
