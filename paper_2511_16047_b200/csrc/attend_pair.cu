@@ -345,7 +345,9 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const uint32_t tiles = (raw + (uint32_t)sizeof(Barriers) + 1023u) & ~1023u;
     const uint32_t q_smem = tiles;
     const uint32_t kv_smem = q_smem + 2 * C::kQBytes;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the warp index is taken through a shuffle so that the compiler knows it to be the same in every
+    // lane: role branches are then uniform branches and the issuing warps keep their operands uniform
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
     const bool layout_ok = (tiles + C::kTileBytes) <= (raw + C::kSmemBytes);
     if (threadIdx.x == 0) {
@@ -511,7 +513,16 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     const uint32_t idesc_s = make_idesc(kQRows, nch * 16, 0);
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
-                        if (!ok || g >= ng) continue;
+                        if (!ok) continue;
+                        if (g >= ng) {
+                            // the stream is absent from this pair: its last P V of the previous pair must not
+                            // wait for a next S that is not coming soon (it also holds a key/value stage)
+                            if (pv_live[g]) {
+                                if (!issue_pv(g)) ok = false;
+                                pv_live[g] = false;
+                            }
+                            continue;
+                        }
                         if (pv_live[g] && !issue_pv(g)) { ok = false; continue; }
                         // S = Q K^T for (stream g, tile j)
                         const uint32_t seq = pp.two_q ? sq : sq + g;

@@ -214,6 +214,22 @@ def test_many_units_per_cta_with_partly_idle_query_tiles(path):
                 check_close(outs[layer][k], want[k], "layer %d scale %d" % (layer, k))
 
 
+@pytest.mark.parametrize("path", [B.PATH_AUTO, B.PATH_TENSOR, B.PATH_TENSOR_PAIR], ids=lambda p: PATH_NAMES[p])
+@pytest.mark.parametrize("D", [64, 128])
+def test_odd_number_of_query_tiles_and_many_key_tiles(path, D):
+    """289 = 2 * 128 + 33 query tokens: three query tiles, so the last pair of every item has a single
+    stream, and enough key/value tiles (6 and more) that a stage held back would stall the ring."""
+    _need(path, D)
+    sides = (4, 17)
+    rows, heads = 10, 40      # 400 items x 2 pairs: several pairs per persistent CTA
+    qkv = make_qkv(rows, heads, sides, D, seed=17)
+    with Cache(1, heads, D, rows, sides, [(0, 9, True)]) as cache:
+        outs = run_pass(cache, qkv, path)
+        want = oracle_outputs(qkv, cache.policies[0], 1.0 / math.sqrt(D))
+        for k in range(len(sides)):
+            check_close(outs[0][k], want[k], "scale %d" % k)
+
+
 def test_full_size_rows_sampled_against_oracle():
     """The VAR-d30 launch shape (512 rows x 30 heads, 680-token schedule) on one cache-efficient and one
     cache-demanding layer; sampled (row, head) items are compared with the oracle at every scale."""
