@@ -41,6 +41,7 @@ constexpr int kThreads = 320;
 constexpr int kMaxStages = 4;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleLog2 = 8.f;
+constexpr int kPolyEvery = 4;     // every 4th pair of exponentials goes to the FMA pipe (0: none)
 
 template <int D>
 struct Cfg {
@@ -130,9 +131,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait; false when it gave up or another role already aborted.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false when it gave up or another role already aborted.  The non-blocking test
+// comes first: most waits here find their phase complete already.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
+    if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 255u) == 255u && *abort_flag) return false;
@@ -288,6 +305,51 @@ __device__ __forceinline__ float fast_exp2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed single-precision pairs (two lanes per instruction on sm_100).
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1)
+{
+    asm("{\n"
+        ".reg .b64 ra, rb, rc, rd;\n"
+        "mov.b64 ra, {%2, %3};\n"
+        "mov.b64 rb, {%4, %5};\n"
+        "mov.b64 rc, {%6, %7};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n"
+        "mov.b64 {%0, %1}, rd;\n"
+        "}\n"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1)
+{
+    asm("{\n"
+        ".reg .b64 ra, rb, rd;\n"
+        "mov.b64 ra, {%2, %3};\n"
+        "mov.b64 rb, {%4, %5};\n"
+        "add.rn.f32x2 rd, ra, rb;\n"
+        "mov.b64 {%0, %1}, rd;\n"
+        "}\n"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+// 2^x for a pair on the FMA pipe instead of the special-function unit: x = n + f with n the
+// nearest integer (obtained by adding 1.5 * 2^23), 2^f by a cubic on [-0.5, 0.5] (relative error
+// below 1e-3, under the bf16 rounding the result gets anyway), and n added into the exponent
+// field.  Inputs below -127 (including -inf) give exactly 0.
+__device__ __forceinline__ void exp2_poly2(float& y0, float& y1, float x0, float x1)
+{
+    constexpr float kMagic = 12582912.f;   // 1.5 * 2^23
+    x0 = fmaxf(x0, -127.f);
+    x1 = fmaxf(x1, -127.f);
+    float r0, r1, n0, n1, f0, f1, p0, p1;
+    add2(r0, r1, x0, x1, kMagic, kMagic);
+    add2(n0, n1, r0, r1, -kMagic, -kMagic);
+    fma2(f0, f1, n0, n1, -1.f, -1.f, x0, x1);
+    fma2(p0, p1, f0, f1, 0.0555041f, 0.0555041f, 0.2402265f, 0.2402265f);
+    fma2(p0, p1, p0, p1, f0, f1, 0.6931472f, 0.6931472f);
+    fma2(p0, p1, p0, p1, f0, f1, 1.f, 1.f);
+    y0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(r0) << 23));
+    y1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(r1) << 23));
+}
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float y;
@@ -386,7 +448,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = bars->tmem_base;
+    const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
     auto tile_of = [&](int j, int32_t& t0, int32_t& valid) {
         if (j < kTileTab) {
             const int2 e = bars->tile_tab[j];
@@ -679,10 +741,17 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
                         for (int i = 0; i < kKT / 4; ++i) {
                             const int c = half * (kKT / 2) + 2 * i;
-                            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), scale_log2, nb));
-                            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), scale_log2, nb));
-                            sum0 += p0;
-                            sum1 += p1;
+                            // every kPolyEvery-th pair takes its exponentials from a polynomial on the FMA pipe:
+                            // the special-function unit (16 results per clock per SM) is the narrowest resource
+                            float x0, x1, p0, p1;
+                            fma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), scale_log2, scale_log2, nb, nb);
+                            if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
+                                exp2_poly2(p0, p1, x0, x1);
+                            } else {
+                                p0 = fast_exp2(x0);
+                                p1 = fast_exp2(x1);
+                            }
+                            add2(sum0, sum1, sum0, sum1, p0, p1);
                             const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                             pk[i] = *reinterpret_cast<const uint32_t*>(&h);
                         }
