@@ -20,6 +20,12 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *  - amskv_append / amskv_attend / amskv_layer_similarity only enqueue work on `stream`:
  *    they allocate nothing, copy nothing between host and device and do not synchronise.
+ *  - Device-side ordering is the caller's when it uses more than one stream.  On one stream the
+ *    calls run in the order made.  With several streams two orders must be kept per layer
+ *    (with events): append(layer, k) before attend(layer, k), and attend(layer, k) before
+ *    append(layer, k + 1), which may overwrite a segment that attend(layer, k) still reads.
+ *    Appends of different layers are independent of each other and of other layers' attends,
+ *    so they can run on a side stream underneath the attention kernels.
  *  - A cache object may be used by one host thread at a time.
  *  - There is no CPU implementation behind any entry point: without a CUDA device the
  *    compute calls fail with AMSKV_ERR_CUDA.

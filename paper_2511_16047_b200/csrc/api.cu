@@ -238,7 +238,8 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
         rc = make_strided(V, strides, cache->heads, T, cache->head_dim, &vs);
         if (rc != AMSKV_OK) return rc;
         cudaError_t e = launch_append(ks, vs, cache->region(layer), lay.offset[scale], T, cache->rows, cache->heads,
-                                      cache->head_dim, static_cast<cudaStream_t>(stream));
+                                      cache->head_dim, cache->status_word(), cache->sm_count,
+                                      static_cast<cudaStream_t>(stream));
         if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
     }
     const int64_t before = scale > 0 ? lay.resident_tokens(cache->tokens, scale - 1) : 0;
