@@ -32,8 +32,10 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0
 
 # DRAM traffic of the attention kernels per step, from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload; filled from the summaries under profiles/.
-NCU_TRAFFIC_BYTES_PER_STEP = {}
+# dram__bytes_write.sum of every attention launch of a 64-row case, scaled by rows and layers:
+# profiles/attention_dram_traffic_var_d30.md), keyed by (workload, policy).  Only valid for the
+# default batch and layer count and for the kernels as they were when it was captured.
+NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams"): 214.6e9}
 
 
 def _peaks():
@@ -149,7 +151,8 @@ def run_ours(args):
 
     def measure(policies, label, instrument, streams=None):
         streams = args.streams if streams is None else streams
-        desc, keep = B.make_desc(wl.layers, wl.heads, wl.head_dim, wl.rows, wl.sides, policies)
+        desc, keep = B.make_desc(wl.layers, wl.heads, wl.head_dim, wl.rows, wl.sides, policies,
+                                 flags=B.FLAG_BULK_APPEND if streams == 2 else 0)
         nbytes = B.amskv_cache_required_bytes(desc)
         free_b, _ = torch.cuda.mem_get_info()
         if nbytes + (2 << 30) > free_b:
@@ -353,7 +356,11 @@ def run_ours(args):
     if rank == 0:
         att_s = main["attend_ms_per_step"] / 1e3
         achieved = main["attend_bytes_per_step"] / att_s / 1e9
-        traffic = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy))
+        traffic = None
+        if not args.batch and not args.layers and args.path == "auto":
+            per_step = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy))
+            if per_step is not None:
+                traffic = round(per_step / (wl.layers * K))   # per attention launch, like `achieved`
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms, 4), "higher_is_better": False, "scaling": "weak",
@@ -374,6 +381,8 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "kernel": "attention (all attend launches of a step)",
                          "achieved": round(achieved, 1), "peak": hbm_gbs, "unit": "GB/s",
                          "frac": round(achieved / hbm_gbs, 4), "peak_kind": peak_kind, "traffic": traffic,
+                         "algorithmic_bytes_per_launch": round(main["attend_bytes_per_step"] / (wl.layers * K)),
+                         "launches_per_step": wl.layers * K,
                          "frac_of_8TBs_nominal": round(achieved / 8000.0, 4)},
             "pass_roofline": {"roofline_ms": round(main["pass_roofline_ms"], 3),
                               "attend_ms": round(main["attend_ms_per_step"], 3),

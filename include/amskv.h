@@ -61,6 +61,13 @@ extern "C" {
                                    attend / similarity are refused; append takes NULL K, V.
                                    For sizing and for inspecting the policy without a GPU. */
 
+#define AMSKV_FLAG_BULK_APPEND 2u /* amskv_append moves token-contiguous inputs with bulk asynchronous
+                                    copies from 32-thread CTAs that need 24 KB of shared memory and
+                                    few registers, so that they fit on an SM beside the attention
+                                    kernel's CTAs.  Meant for callers that enqueue appends on a side
+                                    stream underneath attention; on its own it is a little slower
+                                    than the default copy kernel. */
+
 /* amskv_set_attend_path */
 #define AMSKV_PATH_AUTO 0   /* small-query kernel for 1-4 query tokens, paired tcgen05 kernel otherwise */
 #define AMSKV_PATH_SIMT 1   /* always the CUDA-core kernel                                     */

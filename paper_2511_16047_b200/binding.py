@@ -19,6 +19,7 @@ OK = 0
 ERR_INVALID, ERR_ORDER, ERR_NOMEM, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = -1, -2, -3, -4, -5, -6
 MAX_SCALES = 32
 FLAG_PLAN_ONLY = 1
+FLAG_BULK_APPEND = 2
 PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_PAIR = 0, 1, 2, 3
 
 

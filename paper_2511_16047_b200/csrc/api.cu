@@ -68,7 +68,7 @@ int check_desc(const amskv_desc* d)
         if (d->scale_sides[i] < 1 || d->scale_sides[i] > 4096) return AMSKV_ERR_INVALID;
     for (int l = 0; l < d->layers; ++l)
         if (d->policy[l].n_condensed < 0 || d->policy[l].n_local < 1) return AMSKV_ERR_INVALID;
-    if ((d->flags & ~AMSKV_FLAG_PLAN_ONLY) != 0) return AMSKV_ERR_INVALID;
+    if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND)) != 0) return AMSKV_ERR_INVALID;
     if (!(d->softmax_scale == d->softmax_scale)) return AMSKV_ERR_INVALID;  // NaN
     return AMSKV_OK;
 }
@@ -238,8 +238,8 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
         rc = make_strided(V, strides, cache->heads, T, cache->head_dim, &vs);
         if (rc != AMSKV_OK) return rc;
         cudaError_t e = launch_append(ks, vs, cache->region(layer), lay.offset[scale], T, cache->rows, cache->heads,
-                                      cache->head_dim, cache->status_word(), cache->sm_count,
-                                      static_cast<cudaStream_t>(stream));
+                                      cache->head_dim, (cache->flags & AMSKV_FLAG_BULK_APPEND) != 0, cache->status_word(),
+                                      cache->sm_count, static_cast<cudaStream_t>(stream));
         if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
     }
     const int64_t before = scale > 0 ? lay.resident_tokens(cache->tokens, scale - 1) : 0;

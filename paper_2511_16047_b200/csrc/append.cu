@@ -105,13 +105,8 @@ append_bulk_kernel(const char* __restrict__ Ksrc, const char* __restrict__ Vsrc,
                      ::"r"(smem_addr(bulk_smem + stage * kBulkChunk)), "l"(src), "r"(bytes), "r"(bar)
                      : "memory");
     };
-    for (int64_t c = 0; c < mine && c < kBulkStages - 1; ++c) issue_load(c);
+    for (int64_t c = 0; c < mine && c < kBulkStages; ++c) issue_load(c);
     for (int64_t c = 0; c < mine; ++c) {
-        // the stage of chunk c + kBulkStages - 1 was last read by the store of chunk c - 1
-        if (c + kBulkStages - 1 < mine) {
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            issue_load(c + kBulkStages - 1);
-        }
         const uint32_t stage = (uint32_t)(c % kBulkStages);
         const uint32_t bar = smem_addr(&full[stage]);
         const uint32_t parity = (uint32_t)((c / kBulkStages) & 1);
@@ -157,6 +152,12 @@ append_bulk_kernel(const char* __restrict__ Ksrc, const char* __restrict__ Vsrc,
                      ::"l"(out), "r"(smem_addr(bulk_smem + stage * kBulkChunk)), "r"(bytes)
                      : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        // refill the stage of the previous chunk once its store has read it (the store just issued may
+        // still be reading its own stage)
+        if (c >= 1 && c - 1 + kBulkStages < mine) {
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            issue_load(c - 1 + kBulkStages);
+        }
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores complete before the CTA's shared memory goes away
 }
@@ -164,7 +165,7 @@ append_bulk_kernel(const char* __restrict__ Ksrc, const char* __restrict__ Vsrc,
 }  // namespace
 
 cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion& region, int32_t token_offset,
-                          int32_t T, int32_t rows, int32_t heads, int32_t D, int* status, int sm_count,
+                          int32_t T, int32_t rows, int32_t heads, int32_t D, bool bulk, int* status, int sm_count,
                           cudaStream_t stream)
 {
     const int64_t total = (int64_t)rows * heads * T * (D / 8);
@@ -172,7 +173,7 @@ cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion&
     const int64_t block_bytes = (int64_t)T * D * 2;
     const bool contiguous = K.token == D && V.token == D && K.head == (int64_t)T * D && V.head == (int64_t)T * D &&
                             K.row == (int64_t)heads * T * D && V.row == (int64_t)heads * T * D;
-    if (contiguous && block_bytes >= 4096 && block_bytes < (1ll << 31)) {
+    if (bulk && contiguous && block_bytes >= 4096 && block_bytes < (1ll << 31)) {
         static bool configured = false;
         if (!configured) {
             cudaError_t e = cudaFuncSetAttribute(append_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmem);

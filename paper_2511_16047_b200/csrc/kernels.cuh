@@ -42,7 +42,7 @@ enum DeviceStatus : int {
 };
 
 cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion& region, int32_t token_offset,
-                          int32_t T, int32_t rows, int32_t heads, int32_t D, int* status, int sm_count,
+                          int32_t T, int32_t rows, int32_t heads, int32_t D, bool bulk, int* status, int sm_count,
                           cudaStream_t stream);
 
 cudaError_t launch_attend_simt(const Strided& Q, const Strided& O, const LayerRegion& region, const RangeList& ranges,

@@ -230,6 +230,24 @@ def test_odd_number_of_query_tiles_and_many_key_tiles(path, D):
             check_close(outs[0][k], want[k], "scale %d" % k)
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_bulk_copy_append_gives_the_same_cache(D):
+    """The bulk-copy form of append (for appends that run underneath attention on a side stream) fills the
+    cache exactly like the default copy kernel: outputs of a whole pass are bit-equal."""
+    _need(B.PATH_AUTO, D)
+    sides = (1, 3, 6, 8, 13)
+    rows, heads = 3, 7
+    qkv = make_qkv(rows, heads, sides, D, seed=23)
+    pols = [(1, 2, False), (1, 2, True)]
+    with Cache(2, heads, D, rows, sides, pols) as a, Cache(2, heads, D, rows, sides, pols, flags=B.FLAG_BULK_APPEND) as b:
+        oa, ob = run_pass(a, qkv), run_pass(b, qkv)
+        for layer in range(2):
+            want = oracle_outputs(qkv, pols[layer], 1.0 / math.sqrt(D))
+            for k in range(len(sides)):
+                assert torch.equal(oa[layer][k], ob[layer][k]), (layer, k)
+                check_close(ob[layer][k], want[k], "bulk append layer %d scale %d" % (layer, k))
+
+
 def test_full_size_rows_sampled_against_oracle():
     """The VAR-d30 launch shape (512 rows x 30 heads, 680-token schedule) on one cache-efficient and one
     cache-demanding layer; sampled (row, head) items are compared with the oracle at every scale."""
