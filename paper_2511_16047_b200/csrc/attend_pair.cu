@@ -41,6 +41,7 @@ constexpr int kThreads = 320;
 constexpr int kMaxStages = 4;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleLog2 = 8.f;
+constexpr int kQSplitRows = 64;   // query tiles of at most this many rows are double-buffered inside their slot
 constexpr int kPolyEvery = 4;     // every 4th pair of exponentials goes to the FMA pipe (0: none)
 
 template <int D>
@@ -62,9 +63,9 @@ struct Cfg {
 constexpr int kTileTab = 256;     // tiles whose (first token, valid tokens) are tabulated in shared memory
 
 struct Barriers {
-    uint64_t q_full[2];
+    uint64_t q_full[2][2];     // [stream][half]: see kQSplitRows
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
-    uint64_t s_full[2], p_full[2], o_full[2], o_free[2];
+    uint64_t s_full[2], p_full[2], o_full[2];
     uint32_t tmem_base;
     int abort_flag;
     int2 tile_tab[kTileTab];
@@ -415,11 +416,11 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     if (threadIdx.x == 0) {
         bars->abort_flag = 0;
         for (int g = 0; g < 2; ++g) {
-            mbar_init(smem_u32(&bars->q_full[g]), 1);
+            mbar_init(smem_u32(&bars->q_full[g][0]), 1);
+            mbar_init(smem_u32(&bars->q_full[g][1]), 1);
             mbar_init(smem_u32(&bars->s_full[g]), 1);
             mbar_init(smem_u32(&bars->p_full[g]), kGroupWarps);
             mbar_init(smem_u32(&bars->o_full[g]), 1);
-            mbar_init(smem_u32(&bars->o_free[g]), kGroupWarps);
         }
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars->kv_full[s]), 1);
@@ -459,9 +460,14 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
     };
 
-    const uint32_t q_full0 = smem_u32(&bars->q_full[0]);
+    const uint32_t q_full0 = smem_u32(&bars->q_full[0][0]);   // [g][half] at + 16 * g + 8 * half
+    // With at most 64 query tokens a query tile fills half of its slot, so the slot holds the tiles of two
+    // consecutive units and the next unit's queries are fetched a whole unit ahead.  The MMA reads 128
+    // rows from wherever the tile starts; what it reads past the tile only reaches dead rows of S.
+    const bool q_split = T <= kQSplitRows;
+    constexpr uint32_t kQHalfSlot = kQSplitRows * 128;   // bytes from the first to the second tile of a slot
     const uint32_t s_full0 = smem_u32(&bars->s_full[0]), p_full0 = smem_u32(&bars->p_full[0]);
-    const uint32_t o_full0 = smem_u32(&bars->o_full[0]), o_free0 = smem_u32(&bars->o_free[0]);
+    const uint32_t o_full0 = smem_u32(&bars->o_full[0]);
     const uint32_t kv_full0 = smem_u32(&bars->kv_full[0]), kv_empty0 = smem_u32(&bars->kv_empty[0]);
 
     // pairs of this CTA: p = blockIdx.x + n * gridDim.x, n = 0 .. my_pairs-1
@@ -540,6 +546,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                  pv_last[2] = {false, false};
             uint32_t tcount[2] = {0, 0};   // tiles issued per stream
             uint32_t ucount[2] = {0, 0};   // units started per stream
+            uint32_t q_half[2] = {0, 0};   // half of the query slot the current unit of each stream uses
             uint32_t sq = 0;
 
             // O (+)= P V : M = 128, N = D channels, K = 16 * nch tokens; P from TMEM (packed over S),
@@ -547,7 +554,8 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             auto issue_pv = [&](const int g) -> bool {
                 const uint32_t t = tcount[g] - 1;  // flat tile index of this stream
                 if (!warp_wait(p_full0 + 8 * g, t & 1u, abort_flag)) return false;
-                if (pv_first[g] && !warp_wait(o_free0 + 8 * g, ((ucount[g] - 1) & 1u) ^ 1u, abort_flag)) return false;
+                // (a unit's first P V overwrites O: every warp of the group arrives on p_full for that tile
+                // only after its epilogue of the previous unit, so O has been read by then)
                 tc_fence_after();
                 const uint32_t v_lo = v_lo0 + pv_stage[g] * kStageLo;
                 const uint32_t p_tmem = tmem + C::kSCol + g * kKT;
@@ -585,19 +593,23 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                             }
                             continue;
                         }
-                        if (pv_live[g] && !issue_pv(g)) { ok = false; continue; }
-                        // S = Q K^T for (stream g, tile j)
+                        // S = Q K^T for (stream g, tile j).  Its operands are waited for first: they have
+                        // almost always landed, and this keeps the two waits out of the P -> P V -> S chain.
                         const uint32_t seq = pp.two_q ? sq : sq + g;
                         const uint32_t stage = seq % C::kStages, use = seq / C::kStages;
                         if (j == 0) {
-                            if (!warp_wait(q_full0 + 8 * g, ucount[g] & 1u, abort_flag)) { ok = false; continue; }
+                            const uint32_t u = ucount[g];
+                            q_half[g] = q_split ? (u & 1u) : 0u;
+                            const uint32_t parity = q_split ? ((u >> 1) & 1u) : (u & 1u);
+                            if (!warp_wait(q_full0 + 16 * g + 8 * q_half[g], parity, abort_flag)) { ok = false; continue; }
                             ++ucount[g];
                         }
                         if (!(pp.two_q && g == 1)) {  // the second stream of a shared tile finds it landed already
                             if (!warp_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) { ok = false; continue; }
                         }
+                        if (pv_live[g] && !issue_pv(g)) { ok = false; continue; }
                         tc_fence_after();
-                        const uint32_t q_lo = q_lo0 + g * kQLo;
+                        const uint32_t q_lo = q_lo0 + g * kQLo + q_half[g] * (kQHalfSlot >> 4);
                         const uint32_t k_lo = k_lo0 + stage * kStageLo;
                         const uint32_t d = tmem + C::kSCol + g * kKT;
                         if (elect_one()) {
@@ -634,21 +646,25 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int r = wq * 32 + lane;  // query row inside the tile = TMEM lane
         const uint32_t s_tmem = tmem + C::kSCol + g * kKT + lane_base;
         const uint32_t o_tmem = tmem + C::kOCol + g * D + lane_base;
-        const uint32_t q_full = q_full0 + 8 * g, s_full = s_full0 + 8 * g, p_full = p_full0 + 8 * g;
-        const uint32_t o_full = o_full0 + 8 * g, o_free = o_free0 + 8 * g;
+        const uint32_t s_full = s_full0 + 8 * g, p_full = p_full0 + 8 * g;
+        const uint32_t o_full = o_full0 + 8 * g;
         const bool q_loader = (wq == 0 && lane == 0);
-        uint32_t q_armed = 0;
+        uint32_t q_armed = 0;     // query tiles requested so far
+        uint32_t q_next_n = 0;    // first pair index not yet searched for a query tile
 
-        // fetch the query tile of the first unit at or after pair index n (first lane of the group only)
-        auto load_q = [&](uint32_t n_from) {
-            for (uint32_t n = n_from; n < my_pairs; ++n) {
-                const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
+        // request the query tile of this stream's next unit not yet requested (first lane of the group only)
+        auto load_next_q = [&]() {
+            for (; q_next_n < my_pairs; ++q_next_n) {
+                const int32_t pair = (int32_t)(blockIdx.x + q_next_n * gridDim.x);
                 const Stream s = stream_of(pp, pair, g);
                 if (!s.valid) continue;
                 const int32_t row = s.item / heads, head = s.item - row * heads;
                 const int32_t valid_rows = min(kQRows, T - s.qt * kQRows);
                 const int qboxes = (valid_rows + kQBoxRows - 1) / kQBoxRows;
-                mbar_expect_tx(q_full, (uint32_t)qboxes * kQBoxRows * D * 2);
+                const uint32_t half = q_split ? (q_armed & 1u) : 0u;
+                const uint32_t bar = q_full0 + 16 * g + 8 * half;
+                const uint32_t dst = q_smem + g * C::kQBytes + half * kQHalfSlot;
+                mbar_expect_tx(bar, (uint32_t)qboxes * kQBoxRows * D * 2);
                 int c[4] = {0, 0, 0, 0};
                 c[qpos.y] = head;
                 c[qpos.z] = row;
@@ -656,14 +672,17 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     c[qpos.x] = s.qt * kQRows + bx * kQBoxRows;
 #pragma unroll
                     for (int h = 0; h < C::kHalves; ++h)
-                        tma_load_4d(q_smem + g * C::kQBytes + h * C::kQHalfBytes + bx * kQBoxRows * 128, &q_map, q_full,
-                                    h * 64, c[1], c[2], c[3]);
+                        tma_load_4d(dst + h * C::kQHalfBytes + bx * kQBoxRows * 128, &q_map, bar, h * 64, c[1], c[2], c[3]);
                 }
                 ++q_armed;
+                ++q_next_n;
                 return;
             }
         };
-        if (q_loader) load_q(0);
+        if (q_loader) {
+            load_next_q();
+            if (q_split) load_next_q();
+        }
 
         uint32_t t = 0;   // flat tile counter of this stream
         uint32_t un = 0;  // units done by this stream
@@ -685,7 +704,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 }
                 tc_fence_after();
                 // the last S of this unit has landed, so its query tile is no longer read
-                if (j == n_tiles - 1 && q_loader) load_q(n + 1);
+                if (j == n_tiles - 1 && q_loader) load_next_q();
                 if (warp_live) {
                     uint32_t sr[kKT];
                     tmem_ld64(s_tmem, sr);
@@ -794,15 +813,17 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(o_free);
+            tc_fence_before();   // orders the reads of O before the arrival on p_full for the next unit's first tile
             ++un;
         }
-        // wind down: a query tile requested but never consumed must land before the CTA exits
-        if (q_loader && q_armed > un) {
-            for (uint32_t i = 0; i < kSpinLimit; ++i)
-                if (mbar_try_wait(q_full, (q_armed - 1) & 1u)) break;
+        // wind down: query tiles requested but never consumed must land before the CTA exits
+        if (q_loader) {
+            for (uint32_t q = un; q < q_armed; ++q) {
+                const uint32_t half = q_split ? (q & 1u) : 0u;
+                const uint32_t parity = q_split ? ((q >> 1) & 1u) : (q & 1u);
+                for (uint32_t i = 0; i < kSpinLimit; ++i)
+                    if (mbar_try_wait(q_full0 + 16 * g + 8 * half, parity)) break;
+            }
         }
     }
 
