@@ -138,6 +138,12 @@ def run_ours(args):
         wl = wl.replace(batch=args.batch)
     if args.layers:
         wl = wl.replace(layers=args.layers)
+    if args.condensed is not None:
+        wl = wl.replace(n_condensed=args.condensed)
+    if args.local is not None:
+        wl = wl.replace(n_local=args.local)
+    if args.demanding_fraction is not None:
+        wl = wl.replace(demanding_fraction=args.demanding_fraction)
     hbm_gbs, tflops, peak_kind = _peaks()
     K = len(wl.sides)
     tok = wl.tokens
@@ -160,7 +166,7 @@ def run_ours(args):
         arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         cache = B.amskv_cache_create(desc, arena, nbytes)
         if args.path != "auto":
-            B.amskv_set_attend_path(cache, {"simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR, "pair": B.PATH_TENSOR_PAIR}[args.path])
+            B.amskv_set_attend_path(cache, {"simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR, "pair": B.PATH_TENSOR_PAIR, "small": B.PATH_SMALL}[args.path])
         work = algorithmic_work(wl, policies)
 
         side = torch.cuda.Stream() if streams == 2 else None
@@ -357,7 +363,8 @@ def run_ours(args):
         att_s = main["attend_ms_per_step"] / 1e3
         achieved = main["attend_bytes_per_step"] / att_s / 1e9
         traffic = None
-        if not args.batch and not args.layers and args.path == "auto":
+        if (not args.batch and not args.layers and args.path == "auto" and args.condensed is None and args.local is None
+                and args.demanding_fraction is None):
             per_step = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy))
             if per_step is not None:
                 traffic = round(per_step / (wl.layers * K))   # per attention launch, like `achieved`
@@ -411,29 +418,40 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def oracle_sample(wl, policies, rows):
-    """Times the oracle, as it stands, on a bounded sample of the workload: `rows` rows of one
-    cache-efficient and one cache-demanding layer, all scales.  Work is linear in rows and layers,
-    so the per-image figure for the whole workload is the layer-weighted sum."""
+def oracle_sample(wl, policies, rows, flop_budget=1.0e12):
+    """Times the oracle, as it stands, on a bounded sample of the workload: up to `rows` rows (and, for
+    the long schedules, a subset of the heads) of one layer of each policy kind, all scales.  The sample
+    is cut down to about `flop_budget` fp64 multiply-adds' worth of work.  Work is exactly linear in
+    rows, heads and layers, so the per-image figure for the whole workload is the scaled, layer-weighted sum."""
     import numpy as np
     import oracle
     from paper_2511_16047_b200 import synth
 
     K = len(wl.sides)
     tok = wl.tokens
-    qkv = [synth.qkv_for_scale(rows, wl.heads, tok[k], wl.head_dim, wl.seed, k, "cpu") for k in range(K)]
+    kinds = {}
+    for pol in policies:
+        kinds.setdefault(pol, 0)
+        kinds[pol] += 1
+    per_item = 0.0   # flops of one (row, head) item over all scales and one layer of each kind
+    for (c, w, dem) in kinds:
+        for k in range(K):
+            per_item += 4.0 * tok[k] * sum(tok[s] for s in _kept(k, c, w, dem)) * wl.head_dim
+    rows = max(2, min(rows, wl.rows))
+    heads = wl.heads
+    while rows > 2 and per_item * rows * heads > flop_budget:
+        rows //= 2
+    while heads > 1 and per_item * rows * heads > flop_budget:
+        heads = (heads + 1) // 2
+    qkv = [synth.qkv_for_scale(rows, heads, tok[k], wl.head_dim, wl.seed, k, "cpu") for k in range(K)]
 
     def items(x):
-        return x.double().reshape(rows * wl.heads, x.shape[2], wl.head_dim).numpy()
+        return x.double().reshape(rows * heads, x.shape[2], wl.head_dim).numpy()
 
     Q = [items(q) for q, _, _ in qkv]
     Ks = [items(k) for _, k, _ in qkv]
     Vs = [items(v) for _, _, v in qkv]
     scale = 1.0 / math.sqrt(wl.head_dim)
-    kinds = {}
-    for pol in policies:
-        kinds.setdefault(pol, 0)
-        kinds[pol] += 1
     total_s = 0.0
     weighted = 0.0
     for pol, count in kinds.items():
@@ -445,9 +463,11 @@ def oracle_sample(wl, policies, rows):
         total_s += dt
         weighted += dt * count
     images = rows / 2.0
-    return {"value": round(weighted * 1e6 / images, 1), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": "%d rows x %d heads, one layer of each policy kind (%d kinds), all %d scales: %.1f s measured; "
-                      "value = layer-weighted extrapolation to %d layers" % (rows, wl.heads, len(kinds), K, total_s, wl.layers),
+    head_scale = wl.heads / float(heads)
+    return {"value": round(weighted * head_scale * 1e6 / images, 1), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "%d rows x %d of %d heads, one layer of each policy kind (%d kinds), all %d scales: %.1f s measured; "
+                      "value = extrapolation (linear in rows, heads, layers) to %d heads and %d layers" % (
+                          rows, heads, wl.heads, len(kinds), K, total_s, wl.heads, wl.layers),
             "measured_s": round(total_s, 2)}
 
 
@@ -492,11 +512,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="var_d30")
     ap.add_argument("--policy", default="ams", choices=["ams", "full"])
-    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "pair"],
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "pair", "small"],
                     help="force one attention kernel for every scale (default: the library chooses per scale)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (images)")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
-    ap.add_argument("--cpu-rows", type=int, default=64, help="rows of the oracle's timed sample")
+    ap.add_argument("--condensed", type=int, default=None, help="override the number of condensed scales")
+    ap.add_argument("--local", type=int, default=None, help="override the local window (scales)")
+    ap.add_argument("--demanding-fraction", type=float, default=None, help="override the share of cache-demanding layers")
+    ap.add_argument("--cpu-rows", type=int, default=256, help="rows of the oracle's timed sample")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--streams", type=int, default=1, choices=[1, 2],
                     help="2: appends on a side stream overlapping attention of other layers; 1: everything in order")

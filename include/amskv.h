@@ -69,10 +69,13 @@ extern "C" {
                                     than the default copy kernel. */
 
 /* amskv_set_attend_path */
-#define AMSKV_PATH_AUTO 0   /* small-query kernel for 1-4 query tokens, paired tcgen05 kernel otherwise */
+#define AMSKV_PATH_AUTO 0   /* CUDA-core kernel for a single query token, warp-per-item kernel for the
+                               other coarse scales (at most 16 queries and 32 retained keys), paired
+                               tcgen05 kernel otherwise                                             */
 #define AMSKV_PATH_SIMT 1   /* always the CUDA-core kernel                                     */
 #define AMSKV_PATH_TENSOR 2 /* always the single-stream tcgen05 kernel                         */
 #define AMSKV_PATH_TENSOR_PAIR 3 /* always the paired tcgen05 kernel (two query tiles per CTA)  */
+#define AMSKV_PATH_SMALL 4  /* the warp-per-item kernel wherever it applies (paired kernel elsewhere) */
 
 typedef struct amskv_cache amskv_cache; /* opaque; owned by the library */
 

@@ -16,7 +16,6 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 constexpr size_t kAlign = 256;
 constexpr size_t kStatusBytes = 256;
-constexpr int kSmallQueryMaxTokens = 4;  // scales with at most this many query tokens use the CUDA-core kernel (measured crossover)
 
 static size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -252,8 +251,8 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
 
 int amskv_set_attend_path(amskv_cache* cache, int path)
 {
-    if (!cache || path < AMSKV_PATH_AUTO || path > AMSKV_PATH_TENSOR_PAIR) return AMSKV_ERR_INVALID;
-    if (path >= AMSKV_PATH_TENSOR && !cache->tc_ready) return AMSKV_ERR_UNSUPPORTED;
+    if (!cache || path < AMSKV_PATH_AUTO || path > AMSKV_PATH_SMALL) return AMSKV_ERR_INVALID;
+    if ((path == AMSKV_PATH_TENSOR || path == AMSKV_PATH_TENSOR_PAIR) && !cache->tc_ready) return AMSKV_ERR_UNSUPPORTED;
     cache->path = path;
     return AMSKV_OK;
 }
@@ -275,15 +274,23 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
     ranges.total = 0;
     for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
     const bool tensor = cache->path == AMSKV_PATH_TENSOR;
-    const bool pair = cache->path == AMSKV_PATH_TENSOR_PAIR ||
-                      (cache->path == AMSKV_PATH_AUTO && cache->tc_ready && T > kSmallQueryMaxTokens);
+    // AUTO: the warp-per-item kernel wherever a scale's retained keys fit its register tile, the paired
+    // tcgen05 kernel elsewhere (the CUDA-core kernel only where tensor maps are unavailable)
+    // (a single query token per item is fastest on the CUDA-core kernel: measured)
+    const bool small = (cache->path == AMSKV_PATH_SMALL || (cache->path == AMSKV_PATH_AUTO && T > 1)) &&
+                       small_supported(T, ranges.total);
+    const bool simt = cache->path == AMSKV_PATH_SIMT || (cache->path == AMSKV_PATH_AUTO && T == 1) || !cache->tc_ready;
+    const bool pair = !small && !simt && !tensor;
     cudaError_t e;
-    if (pair) {
+    if (small) {
+        e = launch_attend_small(q, o, cache->region(layer), ranges, T, cache->rows, cache->heads, cache->head_dim,
+                                cache->softmax_scale, static_cast<cudaStream_t>(stream));
+    } else if (pair) {
         e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes,
                                cache->k_maps64[layer].bytes, cache->v_maps64[layer].bytes, ranges, T, cache->rows,
                                cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
                                cache->sm_count, static_cast<cudaStream_t>(stream));
-    } else if (tensor) {
+    } else if (tensor && cache->tc_ready) {
         e = launch_attend_tc(q, o, cache->region(layer), cache->k_maps[layer].bytes, cache->v_maps[layer].bytes, ranges,
                              T, cache->rows, cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
                              cache->sm_count, static_cast<cudaStream_t>(stream));

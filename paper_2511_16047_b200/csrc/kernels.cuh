@@ -73,6 +73,14 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
                                const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
                                float softmax_scale, int* status, int sm_count, cudaStream_t stream);
 
+// Warp-per-item kernel for the coarse scales: every retained key in one register tile.
+constexpr int kSmallMaxKeys = 32;
+constexpr int kSmallMaxQueries = 16;
+bool small_supported(int32_t T, int32_t total_keys);
+cudaError_t launch_attend_small(const Strided& Q, const Strided& O, const LayerRegion& region, const RangeList& ranges,
+                                int32_t T, int32_t rows, int32_t heads, int32_t D, float softmax_scale,
+                                cudaStream_t stream);
+
 void count_launch(int n = 1);
 
 }  // namespace amskv

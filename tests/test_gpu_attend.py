@@ -13,12 +13,12 @@ from gpu_common import (Cache, check_close, make_qkv, oracle_outputs, run_pass, 
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [B.PATH_SIMT, B.PATH_AUTO, B.PATH_TENSOR, B.PATH_TENSOR_PAIR]
-PATH_NAMES = {B.PATH_SIMT: "simt", B.PATH_AUTO: "auto", B.PATH_TENSOR: "tensor", B.PATH_TENSOR_PAIR: "pair"}
+PATHS = [B.PATH_SIMT, B.PATH_AUTO, B.PATH_TENSOR, B.PATH_TENSOR_PAIR, B.PATH_SMALL]
+PATH_NAMES = {B.PATH_SIMT: "simt", B.PATH_AUTO: "auto", B.PATH_TENSOR: "tensor", B.PATH_TENSOR_PAIR: "pair", B.PATH_SMALL: "small"}
 
 
 def _need(path, head_dim=64):
-    if path in (B.PATH_TENSOR, B.PATH_TENSOR_PAIR) and not tensor_path_available(head_dim):
+    if path in (B.PATH_TENSOR, B.PATH_TENSOR_PAIR, B.PATH_SMALL) and not tensor_path_available(head_dim):
         pytest.skip("tensor-core path not available for head_dim %d" % head_dim)
 
 
