@@ -504,6 +504,72 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_similarity(args):
+    """Inter-scale key similarity (Eq. 4) over every adjacent scale pair of every layer of the workload:
+    GB/s against the HBM peak, and the layer classification it yields on seeded correlated /
+    independent layers.  One JSON line; not the headline metric."""
+    import torch
+    from paper_2511_16047_b200 import binding as B
+    from paper_2511_16047_b200 import synth
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    wl = synth.WORKLOADS[args.workload]
+    if args.batch:
+        wl = wl.replace(batch=args.batch)
+    hbm_gbs, _, peak_kind = _peaks()
+    # two key sets per scale: scales share a smooth field with weight 0.9 ("correlated") or 0 ("independent")
+    keys = {rho: synth.smooth_field_keys(wl.rows, wl.heads, wl.sides, wl.head_dim, wl.seed + int(rho * 10), rho, "cuda")
+            for rho in (0.9, 0.0)}
+    n_ws = B.amskv_similarity_workspace_bytes()
+    ws = torch.empty(n_ws, dtype=torch.uint8, device="cuda")
+    mask = wl.demanding_mask()   # demanding layers get the independent keys: low similarity
+    K = len(wl.sides)
+    out = torch.zeros((wl.layers, K - 1), dtype=torch.float64, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for layer in range(wl.layers):
+            ks = keys[0.0 if mask[layer] else 0.9]
+            for i in range(1, K):
+                B.amskv_layer_similarity(ks[i - 1], wl.sides[i - 1], ks[i], wl.sides[i], wl.rows, wl.heads, wl.head_dim,
+                                         out[layer, i - 1:], ws, n_ws, stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    l0 = B.amskv_launch_count()
+    step()
+    launches = B.amskv_launch_count() - l0
+    graph = torch.cuda.CUDAGraph()     # 540 small launches per pass: replayed from a graph like the attention pass
+    with torch.cuda.graph(graph):
+        stream = torch.cuda.current_stream()
+        step()
+    stream = torch.cuda.current_stream()
+    graph.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        graph.replay()
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    tok = wl.tokens
+    bytes_step = wl.layers * sum(2 * wl.rows * wl.heads * wl.head_dim * (tok[i] + tok[i - 1]) for i in range(1, K))
+    scores = (-(out.sum(dim=1)).sqrt()).tolist()     # S = -sqrt(sum of squares over all pairs)
+    chosen = B.amskv_classify_lowest(scores, wl.n_demanding())
+    print(json.dumps({"metric": "inter-scale key similarity, all adjacent pairs of all layers", "value": round(ms, 4), "unit": "ms/pass",
+                      "higher_is_better": False, "n_gpus": 1, "steps": args.steps, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "%s: %d layers, %d rows x %d heads x %d, %d scale pairs per layer; keys larger than L2 at the "
+                                             "large scales" % (wl.name, wl.layers, wl.rows, wl.heads, wl.head_dim, K - 1)},
+                      "gpu_launches": launches * args.steps,
+                      "roofline": {"bound": "hbm", "achieved": round(bytes_step / ms / 1e6, 1), "peak": hbm_gbs, "unit": "GB/s",
+                                   "frac": round(bytes_step / ms / 1e6 / hbm_gbs, 4), "peak_kind": peak_kind, "traffic": None,
+                                   "algorithmic_bytes_per_pass": bytes_step},
+                      "classification": {"lowest_similarity_layers_equal_seeded_independent_layers": chosen == mask}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -523,6 +589,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--streams", type=int, default=1, choices=[1, 2],
                     help="2: appends on a side stream overlapping attention of other layers; 1: everything in order")
+    ap.add_argument("--similarity", action="store_true", help="time amskv_layer_similarity instead of the attention pass")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compare", action="store_true")
@@ -531,6 +598,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.similarity:
+        run_similarity(args)
     else:
         run_ours(args)
 

@@ -50,43 +50,66 @@ __device__ __forceinline__ void tap(int i, float ratio, int s_in, int& i0, int& 
     w = f - (float)i0;
 }
 
-template <int D>
+// Index is uint32_t whenever the chunk count allows it: the per-chunk index arithmetic (two divisions by
+// run-time values) is what this kernel spends its instructions on, and 64-bit division costs several
+// times the 32-bit one.
+template <int D, typename Index>
 __global__ void __launch_bounds__(kThreads)
 similarity_partial_kernel(const uint4* __restrict__ K_prev, int32_t s_prev, const uint4* __restrict__ K_cur,
-                          int32_t s_cur, int64_t total_chunks, double* __restrict__ partials)
+                          int32_t s_cur, int64_t total_chunks_, double* __restrict__ partials)
 {
+    const Index total_chunks = (Index)total_chunks_;
     constexpr int CPT = D / 8;
     __shared__ double smem[kThreads / 32];
     const float ratio = (float)s_prev / (float)s_cur;
     const int32_t t_cur = s_cur * s_cur, t_prev = s_prev * s_prev;
     double acc = 0.0;
-    for (int64_t idx = (int64_t)blockIdx.x * kThreads + threadIdx.x; idx < total_chunks;
-         idx += (int64_t)gridDim.x * kThreads) {
-        const int64_t tok_global = idx / CPT;
-        const int32_t ch = (int32_t)(idx - tok_global * CPT);
-        const int64_t item = tok_global / t_cur;
-        const int32_t tok = (int32_t)(tok_global - item * t_cur);
-        const int32_t y = tok / s_cur, x = tok - y * s_cur;
-        int y0, y1, x0, x1;
-        float wy, wx;
-        tap(y, ratio, s_prev, y0, y1, wy);
-        tap(x, ratio, s_prev, x0, x1, wx);
-        const uint4* P = K_prev + item * (int64_t)t_prev * CPT + ch;
-        float c[8], v00[8], v01[8], v10[8], v11[8];
-        unpack8(__ldcs(K_cur + idx), c);
-        unpack8(__ldg(P + (int64_t)(y0 * s_prev + x0) * CPT), v00);
-        unpack8(__ldg(P + (int64_t)(y0 * s_prev + x1) * CPT), v01);
-        unpack8(__ldg(P + (int64_t)(y1 * s_prev + x0) * CPT), v10);
-        unpack8(__ldg(P + (int64_t)(y1 * s_prev + x1) * CPT), v11);
-        float part = 0.f;
+    // Two chunks per thread and iteration, all ten loads issued before either is used: a thread's one
+    // 16-byte HBM load per iteration would leave the memory system a third full.
+    constexpr int kPer = 2;
+    const Index stride = (Index)gridDim.x * kThreads;
+    for (Index base = (Index)blockIdx.x * kThreads + threadIdx.x; base < total_chunks; base += kPer * stride) {
+        uint4 cur[kPer], t00[kPer], t01[kPer], t10[kPer], t11[kPer];
+        float wy[kPer], wx[kPer];
+        bool live[kPer];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float top = v00[i] + wx * (v01[i] - v00[i]);
-            const float bot = v10[i] + wx * (v11[i] - v10[i]);
-            const float diff = c[i] - (top + wy * (bot - top));
-            part = fmaf(diff, diff, part);
+        for (int u = 0; u < kPer; ++u) {
+            const Index idx = base + (Index)u * stride;
+            live[u] = idx < total_chunks && idx >= base;   // (the second test catches wrap-around of a narrow index)
+            const Index safe = live[u] ? idx : base;
+            const Index tok_global = safe / CPT;
+            const int32_t ch = (int32_t)(safe - tok_global * CPT);
+            const Index item = tok_global / (Index)t_cur;
+            const int32_t tok = (int32_t)(tok_global - item * (Index)t_cur);
+            const int32_t y = tok / s_cur, x = tok - y * s_cur;
+            int y0, y1, x0, x1;
+            tap(y, ratio, s_prev, y0, y1, wy[u]);
+            tap(x, ratio, s_prev, x0, x1, wx[u]);
+            const uint4* P = K_prev + (int64_t)item * t_prev * CPT + ch;
+            cur[u] = __ldcs(K_cur + safe);
+            t00[u] = __ldg(P + (int64_t)(y0 * s_prev + x0) * CPT);
+            t01[u] = __ldg(P + (int64_t)(y0 * s_prev + x1) * CPT);
+            t10[u] = __ldg(P + (int64_t)(y1 * s_prev + x0) * CPT);
+            t11[u] = __ldg(P + (int64_t)(y1 * s_prev + x1) * CPT);
         }
-        acc += (double)part;
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            float c[8], v00[8], v01[8], v10[8], v11[8];
+            unpack8(cur[u], c);
+            unpack8(t00[u], v00);
+            unpack8(t01[u], v01);
+            unpack8(t10[u], v10);
+            unpack8(t11[u], v11);
+            float part = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float top = v00[i] + wx[u] * (v01[i] - v00[i]);
+                const float bot = v10[i] + wx[u] * (v11[i] - v10[i]);
+                const float diff = c[i] - (top + wy[u] * (bot - top));
+                part = fmaf(diff, diff, part);
+            }
+            if (live[u]) acc += (double)part;
+        }
     }
     const double total = block_sum(acc, smem);
     if (threadIdx.x == 0) partials[blockIdx.x] = total;
@@ -112,12 +135,16 @@ cudaError_t launch_similarity(const __nv_bfloat16* K_prev, int32_t side_prev, co
     int64_t blocks = (total + kThreads - 1) / kThreads;
     if (blocks > kSimilarityMaxBlocks) blocks = kSimilarityMaxBlocks;
     if (blocks < 1) blocks = 1;
+    // the grid-stride loop adds gridDim * kThreads to an index below total: keep that sum inside 32 bits
+    const bool narrow = total + 2ll * kSimilarityMaxBlocks * kThreads < (1ll << 32);
+    const uint4* kp = (const uint4*)K_prev;
+    const uint4* kc = (const uint4*)K_cur;
     if (D == 64) {
-        similarity_partial_kernel<64><<<(unsigned)blocks, kThreads, 0, stream>>>(
-            (const uint4*)K_prev, side_prev, (const uint4*)K_cur, side_cur, total, partials);
+        if (narrow) similarity_partial_kernel<64, uint32_t><<<(unsigned)blocks, kThreads, 0, stream>>>(kp, side_prev, kc, side_cur, total, partials);
+        else similarity_partial_kernel<64, int64_t><<<(unsigned)blocks, kThreads, 0, stream>>>(kp, side_prev, kc, side_cur, total, partials);
     } else {
-        similarity_partial_kernel<128><<<(unsigned)blocks, kThreads, 0, stream>>>(
-            (const uint4*)K_prev, side_prev, (const uint4*)K_cur, side_cur, total, partials);
+        if (narrow) similarity_partial_kernel<128, uint32_t><<<(unsigned)blocks, kThreads, 0, stream>>>(kp, side_prev, kc, side_cur, total, partials);
+        else similarity_partial_kernel<128, int64_t><<<(unsigned)blocks, kThreads, 0, stream>>>(kp, side_prev, kc, side_cur, total, partials);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
