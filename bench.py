@@ -32,8 +32,8 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0
 
 # DRAM traffic of the attention kernels per step, from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of every attention launch of a 64-row case, scaled by rows and layers:
-# profiles/attention_dram_traffic_var_d30.md), keyed by (workload, policy).  Only valid for the
+# dram__bytes_write.sum of every attention launch of a 64-row case, scaled by rows and layers; the
+# capture is summarised under profiles/), keyed by (workload, policy).  Only valid for the
 # default batch and layer count and for the kernels as they were when it was captured.
 NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams"): 214.6e9}
 

@@ -130,7 +130,12 @@ def similarity_ss(K_prev, s_prev: int, K_cur, s_cur: int) -> float:
 
 
 def similarity(K_prev, s_prev: int, K_cur, s_cur: int) -> float:
-    """Eq. 4: S(k_i, k-hat_{i-1}) = -|| k_i - k-hat_{i-1} ||_2 over all items/tokens/channels."""
+    """Eq. 4: S(k_i, k-hat_{i-1}) = -|| k_i - k-hat_{i-1} ||_2 over all items/tokens/channels.
+
+    The arithmetic of this reading (bilinear resize, half-pixel centres, edge clamp, plain L2 norm) is
+    pinned by the tests.  Parity unpinned: the paper's threshold values (around -0.01, Appendix E) imply
+    a normalisation of the norm that the text does not state, and its per-layer values exist only as a
+    figure, so nothing ties the magnitude of this score to the paper's."""
     return -float(np.sqrt(similarity_ss(K_prev, s_prev, K_cur, s_cur)))
 
 
