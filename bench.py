@@ -52,14 +52,19 @@ def _kept(k, c, w, dem):
     return [s for s in range(k + 1) if dem or s < c or s > k - w]
 
 
-def algorithmic_work(wl, policies):
-    """Per (layer, scale): bytes = Q read + out write + kept K,V read once; flops = 4 T L D per item."""
+def algorithmic_work(wl, policies, budgets=None, cache=None):
+    """Per (layer, scale): bytes = Q read + out write + kept K,V read once; flops = 4 T L D per item.
+    Under token budgets the attended key count comes from the library's host-side plan."""
+    from paper_2511_16047_b200 import binding as B
     items = wl.rows * wl.heads
     tok = wl.tokens
     per = {}
     for layer, (c, w, dem) in enumerate(policies):
         for k in range(len(tok)):
-            L = sum(tok[s] for s in _kept(k, c, w, dem))
+            if budgets is not None and budgets[layer][0] > 0:
+                L = sum(n for _, _, n in B.amskv_attended_tokens(cache, layer, k))
+            else:
+                L = sum(tok[s] for s in _kept(k, c, w, dem))
             per[(layer, k)] = (2 * wl.head_dim * items * (2 * tok[k] + 2 * L), 4 * tok[k] * L * wl.head_dim * items)
     return per
 
@@ -155,10 +160,10 @@ def run_ours(args):
     outs = [torch.empty_like(q) for q, _, _ in qkv]
     input_bytes = sum(3 * q.numel() * 2 for q, _, _ in qkv)
 
-    def measure(policies, label, instrument, streams=None):
+    def measure(policies, label, instrument, streams=None, budgets=None):
         streams = args.streams if streams is None else streams
         desc, keep = B.make_desc(wl.layers, wl.heads, wl.head_dim, wl.rows, wl.sides, policies,
-                                 flags=B.FLAG_BULK_APPEND if streams == 2 else 0)
+                                 flags=B.FLAG_BULK_APPEND if streams == 2 else 0, token_budgets=budgets)
         nbytes = B.amskv_cache_required_bytes(desc)
         free_b, _ = torch.cuda.mem_get_info()
         if nbytes + (2 << 30) > free_b:
@@ -167,7 +172,7 @@ def run_ours(args):
         cache = B.amskv_cache_create(desc, arena, nbytes)
         if args.path != "auto":
             B.amskv_set_attend_path(cache, {"simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR, "pair": B.PATH_TENSOR_PAIR, "small": B.PATH_SMALL}[args.path])
-        work = algorithmic_work(wl, policies)
+        work = algorithmic_work(wl, policies, budgets, cache)
 
         side = torch.cuda.Stream() if streams == 2 else None
         n_ev = wl.layers * K
@@ -280,7 +285,8 @@ def run_ours(args):
         return result
 
     policies = wl.policies(full_retention=args.policy == "full")
-    main = measure(policies, args.policy, instrument=True)
+    budgets = wl.token_budgets() if args.policy == "tokens" else None
+    main = measure(policies, args.policy, instrument=True, budgets=budgets)
     if "skipped" in main:
         raise SystemExit("workload does not fit: " + main["skipped"])
     cache, arena, desc, keep = main.pop("_cache")
@@ -329,7 +335,7 @@ def run_ours(args):
     # the same pass with the appends on a side stream (they then overlap other layers' attention)
     overlap = None
     if not args.no_compare and args.streams == 1:
-        overlap = measure(policies, args.policy + ", two streams", instrument=False, streams=2)
+        overlap = measure(policies, args.policy + ", two streams", instrument=False, streams=2, budgets=budgets)
         if "_cache" in overlap:
             c3, a3, _, _ = overlap.pop("_cache")
             B.amskv_cache_destroy(c3)
@@ -339,7 +345,7 @@ def run_ours(args):
     # the other policy (full retention when timing AMS-KV and vice versa): KV bytes and latency beside it
     other = None
     if not args.no_compare:
-        other_name = "full" if args.policy == "ams" else "ams"
+        other_name = "ams" if args.policy == "full" else "full"
         other = measure(wl.policies(full_retention=other_name == "full"), other_name, instrument=False)
         if "_cache" in other:
             c2, a2, _, _ = other.pop("_cache")
@@ -357,7 +363,7 @@ def run_ours(args):
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = oracle_sample(wl, policies, args.cpu_rows)
+        cpu_baseline = oracle_sample(wl, policies, args.cpu_rows, budgets=budgets)
 
     if rank == 0:
         att_s = main["attend_ms_per_step"] / 1e3
@@ -418,7 +424,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def oracle_sample(wl, policies, rows, flop_budget=1.0e12):
+def oracle_sample(wl, policies, rows, flop_budget=1.0e12, budgets=None):
     """Times the oracle, as it stands, on a bounded sample of the workload: up to `rows` rows (and, for
     the long schedules, a subset of the heads) of one layer of each policy kind, all scales.  The sample
     is cut down to about `flop_budget` fp64 multiply-adds' worth of work.  Work is exactly linear in
@@ -430,13 +436,23 @@ def oracle_sample(wl, policies, rows, flop_budget=1.0e12):
     K = len(wl.sides)
     tok = wl.tokens
     kinds = {}
-    for pol in policies:
+    for layer, pol in enumerate(policies):
+        if budgets is not None and budgets[layer][0] > 0:
+            pol = ("tokens",) + tuple(budgets[layer])
         kinds.setdefault(pol, 0)
         kinds[pol] += 1
+
+    def attended(pol, k):
+        """Keys of scale k's queries: segment ids (whole scales) or a (segment, token) list (token budgets)."""
+        if pol[0] == "tokens":
+            return oracle.attended_tokens(wl.sides, k, pol[1], pol[2])
+        return oracle.keep_set(k, pol[0], pol[1], pol[2])
+
     per_item = 0.0   # flops of one (row, head) item over all scales and one layer of each kind
-    for (c, w, dem) in kinds:
+    for pol in kinds:
         for k in range(K):
-            per_item += 4.0 * tok[k] * sum(tok[s] for s in _kept(k, c, w, dem)) * wl.head_dim
+            L = len(attended(pol, k)) if pol[0] == "tokens" else sum(tok[s] for s in attended(pol, k))
+            per_item += 4.0 * tok[k] * L * wl.head_dim
     rows = max(2, min(rows, wl.rows))
     heads = wl.heads
     while rows > 2 and per_item * rows * heads > flop_budget:
@@ -455,10 +471,12 @@ def oracle_sample(wl, policies, rows, flop_budget=1.0e12):
     total_s = 0.0
     weighted = 0.0
     for pol, count in kinds.items():
-        c, w, dem = pol
         t0 = time.perf_counter()
         for k in range(K):
-            oracle.attend_selected(Q[k], Ks, Vs, oracle.keep_set(k, c, w, dem), scale)
+            if pol[0] == "tokens":
+                oracle.attend_tokens(Q[k], Ks, Vs, attended(pol, k), scale)
+            else:
+                oracle.attend_selected(Q[k], Ks, Vs, attended(pol, k), scale)
         dt = time.perf_counter() - t0
         total_s += dt
         weighted += dt * count
@@ -483,13 +501,14 @@ def run_reference(args):
     if args.layers:
         wl = wl.replace(layers=args.layers)
     policies = wl.policies(full_retention=args.policy == "full")
+    budgets = wl.token_budgets() if args.policy == "tokens" else None
     rows = max(2, args.cpu_rows // 4)
     for _ in range(max(1, min(args.warmup, 1))):
-        oracle_sample(wl, policies, 2)
+        oracle_sample(wl, policies, 2, budgets=budgets)
     vals, secs = [], 0.0
     steps = max(1, min(args.steps, 3))
     for _ in range(steps):
-        r = oracle_sample(wl, policies, rows)
+        r = oracle_sample(wl, policies, rows, budgets=budgets)
         vals.append(r["value"])
         secs += r["measured_s"]
     value = sum(vals) / len(vals)
@@ -577,7 +596,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="var_d30")
-    ap.add_argument("--policy", default="ams", choices=["ams", "full"])
+    ap.add_argument("--policy", default="ams", choices=["ams", "full", "tokens"],
+                    help="ams: whole scales (condensed + local window); full: every scale; tokens: Algorithm 1 "
+                         "and 2 with token budgets (C_cds = the condensed scales, C_min = C_cds + the penultimate "
+                         "scale, C_max = C_cds + the last two scales)")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "pair", "small"],
                     help="force one attention kernel for every scale (default: the library chooses per scale)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (images)")

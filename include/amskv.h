@@ -94,6 +94,29 @@ typedef struct {
     int32_t cache_demanding;
 } amskv_layer_policy;
 
+/*
+ * Per-layer token budget: Algorithm 1 with Algorithm 2 (Appendix F) as its roll, taken literally,
+ * with capacities counted in tokens (Sec. 5 sets C_max to the condensed scales plus the last two
+ * scales and C_min to the condensed scales plus the penultimate one).
+ *   budget_tokens     C_bgt > 0: the layer holds at most this many tokens per (row, head).  Pass
+ *                     C_max for a cache-demanding layer and C_min for a cache-efficient one:
+ *                     nothing is evicted before a layer's first overflow, so starting at C_max
+ *                     equals Algorithm 1's promotion at that overflow.  0 = this layer follows
+ *                     its amskv_layer_policy (whole scales) instead.
+ *   condensed_tokens  C_cds >= 0 in tokens (clamped to the budget): the first C_cds cached
+ *                     tokens are pinned.
+ * After the append of a scale the cache holds every cached token while their number is within
+ * the budget, else the first C_cds of them and the most recent C_bgt - C_cds: the tail may end
+ * inside a scale.  A scale with more tokens than the budget is never cached (Algorithm 1 skips
+ * it).  The queries of a scale always attend to that whole scale besides the cache (the paper
+ * leaves this open; without it the skipped scale would not see itself): a scale that is not
+ * resident in full after its own append is kept in a transient slot until the next append.
+ */
+typedef struct {
+    int32_t budget_tokens;
+    int32_t condensed_tokens;
+} amskv_token_budget;
+
 typedef struct {
     int32_t layers;
     int32_t heads;
@@ -104,6 +127,7 @@ typedef struct {
     const amskv_layer_policy* policy; /* [layers]; copied                                  */
     float softmax_scale;         /* <= 0 selects 1/sqrt(head_dim)                          */
     uint32_t flags;              /* AMSKV_FLAG_*                                           */
+    const amskv_token_budget* token_budget; /* [layers] or NULL (no layer uses token budgets); copied */
 } amskv_desc;
 
 /* Bytes of device memory a cache for `desc` needs (its KV arena; Appendix D, Eq. 5 counts
@@ -221,16 +245,33 @@ AMSKV_API int amskv_classify_by_threshold(const double* scores, int layers, doub
 AMSKV_API int amskv_classify_lowest(const double* scores, int layers, int n_demanding, int32_t* demanding);
 
 /* Segment ids `layer` retains right after scale `scale` was appended, ascending (host-only;
- * a pure function of the policy).  ids must hold AMSKV_MAX_SCALES entries. */
+ * a pure function of the policy).  ids must hold AMSKV_MAX_SCALES entries.  Under a token budget a
+ * segment counts as retained while the cache holds at least one of its tokens. */
 AMSKV_API int amskv_kept_segments(const amskv_cache* cache, int layer, int scale, int32_t* ids, int32_t* n);
 
-/* Segment ids the append of `scale` drops from `layer` (host-only). */
+/* Segment ids the append of `scale` drops from `layer` (host-only).  Under a token budget: the
+ * segments that lose their last cached token; a scale too large to be cached is reported at its own
+ * step. */
 AMSKV_API int amskv_evicted_at(const amskv_cache* cache, int layer, int scale, int32_t* ids, int32_t* n);
 
 /* Token ranges (start, length) of the layer's per-(row, head) arena region that attend
  * reads at `scale`, merged where adjacent (host-only).  ranges must hold
  * 2 * AMSKV_MAX_SCALES entries. */
 AMSKV_API int amskv_resident_ranges(const amskv_cache* cache, int layer, int scale, int32_t* ranges, int32_t* n);
+
+/* The keys the queries of `scale` attend to in `layer`, as runs (segment, first token, count) in
+ * ascending segment order (host-only; a pure function of the policy).  Whole segments under the
+ * scale-granular policy; under a token budget a segment may appear with part of its tokens, as up to
+ * two runs (its share of the pinned head and of the tail).  runs must hold 3 * 2 * AMSKV_MAX_SCALES
+ * entries; *n receives the number of runs. */
+AMSKV_API int amskv_attended_tokens(const amskv_cache* cache, int layer, int scale, int32_t* runs, int32_t* n);
+
+/* The copies amskv_append(layer, scale) performs, as triples (first source token, destination
+ * position in the per-(row, head) region, tokens) (host-only).  One copy under the scale-granular
+ * policy; up to AMSKV_MAX_APPEND_COPIES under a token budget (pinned head, the ring's two sides of
+ * its wrap point, transient slot).  copies must hold 3 * AMSKV_MAX_APPEND_COPIES entries. */
+#define AMSKV_MAX_APPEND_COPIES 4
+AMSKV_API int amskv_append_copies(const amskv_cache* cache, int layer, int scale, int32_t* copies, int32_t* n);
 
 /* Bytes: the arena, the KV bytes resident now, and the largest residency seen since the
  * last reset. */

@@ -16,8 +16,8 @@ from typing import List, Sequence
 
 import numpy as np
 
-from .selection import (algorithm1_tokens, clru_tokens, evicted_at, keep_set,  # noqa: F401
-                        keep_set_simulated, kept_tokens, kv_bytes)
+from .selection import (algorithm1_tokens, attended_tokens, clru_tokens, evicted_at,  # noqa: F401
+                        keep_set, keep_set_simulated, kept_tokens, kv_bytes)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "amskv_oracle.c")
@@ -94,6 +94,24 @@ def attend_selected(Q, K_segments: Sequence, V_segments: Sequence, keep: Sequenc
     Kc = np.concatenate([_f64(K_segments[s]) for s in keep], axis=1)
     Vc = np.concatenate([_f64(V_segments[s]) for s in keep], axis=1)
     return attention(Q, Kc, Vc, scale)
+
+
+def attend_tokens(Q, K_segments: Sequence, V_segments: Sequence, tokens: Sequence, scale: float) -> np.ndarray:
+    """Attention of Q over an explicit list of (segment, token) keys (token budgets may keep part
+    of a segment).  K_segments[s], V_segments[s]: [n, T_s, D]."""
+    tokens = list(tokens)
+    k_parts, v_parts = [], []
+    i = 0
+    while i < len(tokens):  # gather run by run of equal segment id, in list order
+        s = tokens[i][0]
+        j = i
+        while j < len(tokens) and tokens[j][0] == s:
+            j += 1
+        idx = [t for _, t in tokens[i:j]]
+        k_parts.append(_f64(K_segments[s])[:, idx, :])
+        v_parts.append(_f64(V_segments[s])[:, idx, :])
+        i = j
+    return attention(Q, np.concatenate(k_parts, axis=1), np.concatenate(v_parts, axis=1), scale)
 
 
 def block_causal_attention(Q_all, K_all, V_all, sides: Sequence[int], scale: float) -> np.ndarray:

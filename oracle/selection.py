@@ -10,7 +10,11 @@ Reading of the paper taken here (the text is ambiguous on the first point):
     tail is the current scale;
   * the scale-granular rule keeps whole scales: `n_condensed` leading scales are pinned and
     the `n_local` most recent scales form the FIFO tail;
-  * a cache-demanding layer keeps every scale (full retention).
+  * a cache-demanding layer keeps every scale (full retention);
+  * with token budgets (Algorithm 1 and 2 taken literally) the queries of a scale attend to the
+    cache as it stands after that scale's step plus every token of the scale itself: the paper
+    does not say what a scale that Algorithm 1 skips, or that its own roll cuts, attends to, and
+    without its own keys it could not see itself.
 """
 from __future__ import annotations
 
@@ -108,6 +112,18 @@ def algorithm1_tokens(sides: Sequence[int], c_min: int, c_max: int, c_cds: int,
         cache = grown
         history.append(list(cache))
     return history
+
+
+def attended_tokens(sides: Sequence[int], k: int, c_bgt: int, c_cds: int) -> List[Tuple[int, int]]:
+    """(scale, token) pairs the queries of scale k attend to in a layer whose budget is fixed at c_bgt.
+
+    The cache Algorithm 1 leaves after scale k (budget c_bgt from the start: see
+    `algorithm1_tokens`, whose promotion happens before anything was evicted), followed by the
+    tokens of scale k that the cache does not hold.
+    """
+    cache = algorithm1_tokens(list(sides[:k + 1]), c_bgt, c_bgt, c_cds, promote_at_overflow=False)[k]
+    have = set(cache)
+    return cache + [(k, t) for t in range(int(sides[k]) ** 2) if (k, t) not in have]
 
 
 def kv_bytes(sides: Sequence[int], policies: Sequence[Tuple[int, int, bool]], rows: int,

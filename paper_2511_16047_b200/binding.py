@@ -27,11 +27,16 @@ class LayerPolicy(ctypes.Structure):
     _fields_ = [("n_condensed", ctypes.c_int32), ("n_local", ctypes.c_int32), ("cache_demanding", ctypes.c_int32)]
 
 
+class TokenBudget(ctypes.Structure):
+    _fields_ = [("budget_tokens", ctypes.c_int32), ("condensed_tokens", ctypes.c_int32)]
+
+
 class Desc(ctypes.Structure):
     _fields_ = [("layers", ctypes.c_int32), ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
                 ("rows", ctypes.c_int32), ("n_scales", ctypes.c_int32),
                 ("scale_sides", ctypes.POINTER(ctypes.c_int32)), ("policy", ctypes.POINTER(LayerPolicy)),
-                ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_uint32)]
+                ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_uint32),
+                ("token_budget", ctypes.POINTER(TokenBudget))]
 
 
 class AmskvError(RuntimeError):
@@ -66,6 +71,8 @@ def _load() -> ctypes.CDLL:
         "amskv_kept_segments": ([vp, i, i, i32p, i32p], i),
         "amskv_evicted_at": ([vp, i, i, i32p, i32p], i),
         "amskv_resident_ranges": ([vp, i, i, i32p, i32p], i),
+        "amskv_attended_tokens": ([vp, i, i, i32p, i32p], i),
+        "amskv_append_copies": ([vp, i, i, i32p, i32p], i),
         "amskv_cache_bytes": ([vp, szp, szp, szp], i),
         "amskv_status": ([vp, ctypes.POINTER(i)], i),
         "amskv_launch_count": ([], ctypes.c_int64),
@@ -82,7 +89,8 @@ lib = _load()
 EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy amskv_cache_reset amskv_append "
            "amskv_attend amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
            "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
-           "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_cache_bytes amskv_status "
+           "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_attended_tokens amskv_append_copies "
+           "amskv_cache_bytes amskv_status "
            "amskv_launch_count amskv_strerror").split()
 
 
@@ -123,12 +131,21 @@ def _stream(stream) -> Optional[int]:
 
 
 def make_desc(layers: int, heads: int, head_dim: int, rows: int, sides: Sequence[int],
-              policies: Sequence[Tuple[int, int, bool]], softmax_scale: float = 0.0, flags: int = 0):
-    """Returns (Desc, keepalive) -- keepalive holds the arrays the descriptor points to."""
+              policies: Sequence[Tuple[int, int, bool]], softmax_scale: float = 0.0, flags: int = 0,
+              token_budgets: Optional[Sequence[Tuple[int, int]]] = None):
+    """Returns (Desc, keepalive) -- keepalive holds the arrays the descriptor points to.
+
+    token_budgets: optional per-layer (budget_tokens, condensed_tokens); a layer with budget 0
+    follows its entry of `policies`."""
     sides_arr = (ctypes.c_int32 * len(sides))(*[int(s) for s in sides])
     pol_arr = (LayerPolicy * len(policies))(*[LayerPolicy(int(c), int(w), 1 if d else 0) for c, w, d in policies])
-    d = Desc(layers, heads, head_dim, rows, len(sides), sides_arr, pol_arr, float(softmax_scale), flags)
-    return d, (sides_arr, pol_arr)
+    bud_arr = None
+    if token_budgets is not None:
+        assert len(token_budgets) == len(policies)
+        bud_arr = (TokenBudget * len(token_budgets))(*[TokenBudget(int(b), int(c)) for b, c in token_budgets])
+    d = Desc(layers, heads, head_dim, rows, len(sides), sides_arr, pol_arr, float(softmax_scale), flags,
+             bud_arr if bud_arr is not None else ctypes.cast(None, ctypes.POINTER(TokenBudget)))
+    return d, (sides_arr, pol_arr, bud_arr)
 
 
 def amskv_cache_required_bytes(desc: Desc) -> int:
@@ -235,6 +252,23 @@ def amskv_evicted_at(cache: int, layer: int, scale: int) -> List[int]:
 def amskv_resident_ranges(cache: int, layer: int, scale: int) -> List[Tuple[int, int]]:
     flat = _ids(lib.amskv_resident_ranges, "amskv_resident_ranges", cache, layer, scale, width=2)
     return [(flat[2 * j], flat[2 * j + 1]) for j in range(len(flat) // 2)]
+
+
+def _triples(fn, where: str, cache: int, layer: int, scale: int) -> List[Tuple[int, int, int]]:
+    buf = (ctypes.c_int32 * (3 * 2 * MAX_SCALES))()
+    n = ctypes.c_int32(0)
+    _check(fn(cache, layer, scale, buf, ctypes.byref(n)), where)
+    return [(int(buf[3 * j]), int(buf[3 * j + 1]), int(buf[3 * j + 2])) for j in range(n.value)]
+
+
+def amskv_attended_tokens(cache: int, layer: int, scale: int) -> List[Tuple[int, int, int]]:
+    """Runs (segment, first token, count) the queries of `scale` attend to."""
+    return _triples(lib.amskv_attended_tokens, "amskv_attended_tokens", cache, layer, scale)
+
+
+def amskv_append_copies(cache: int, layer: int, scale: int) -> List[Tuple[int, int, int]]:
+    """Copies (first source token, destination position, tokens) that append(layer, scale) performs."""
+    return _triples(lib.amskv_append_copies, "amskv_append_copies", cache, layer, scale)
 
 
 def amskv_cache_bytes(cache: int) -> Tuple[int, int, int]:

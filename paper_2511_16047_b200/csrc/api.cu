@@ -65,8 +65,13 @@ int check_desc(const amskv_desc* d)
     if (d->head_dim != 64 && d->head_dim != 128) return AMSKV_ERR_UNSUPPORTED;
     for (int i = 0; i < d->n_scales; ++i)
         if (d->scale_sides[i] < 1 || d->scale_sides[i] > 4096) return AMSKV_ERR_INVALID;
-    for (int l = 0; l < d->layers; ++l)
+    for (int l = 0; l < d->layers; ++l) {
+        if (d->token_budget && d->token_budget[l].budget_tokens != 0) {
+            if (d->token_budget[l].budget_tokens < 0 || d->token_budget[l].condensed_tokens < 0) return AMSKV_ERR_INVALID;
+            continue;  // the layer's scale-granular fields are not used
+        }
         if (d->policy[l].n_condensed < 0 || d->policy[l].n_local < 1) return AMSKV_ERR_INVALID;
+    }
     if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND)) != 0) return AMSKV_ERR_INVALID;
     if (!(d->softmax_scale == d->softmax_scale)) return AMSKV_ERR_INVALID;  // NaN
     return AMSKV_OK;
@@ -93,7 +98,10 @@ int plan(const amskv_desc* d, amskv_cache* c)
     c->layer_offset.resize(d->layers);
     size_t at = kStatusBytes;
     for (int l = 0; l < d->layers; ++l) {
-        c->layout[l].build(c->tokens, d->policy[l].n_condensed, d->policy[l].n_local, d->policy[l].cache_demanding != 0);
+        if (d->token_budget && d->token_budget[l].budget_tokens > 0)
+            c->layout[l].build_tokens(c->tokens, d->token_budget[l].budget_tokens, d->token_budget[l].condensed_tokens);
+        else
+            c->layout[l].build(c->tokens, d->policy[l].n_condensed, d->policy[l].n_local, d->policy[l].cache_demanding != 0);
         if ((int64_t)c->layout[l].capacity > (1ll << 30)) return AMSKV_ERR_INVALID;
         c->layer_offset[l] = at;
         at += align_up((size_t)c->layout[l].capacity * c->token_bytes());
@@ -236,10 +244,17 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
         if (rc != AMSKV_OK) return rc;
         rc = make_strided(V, strides, cache->heads, T, cache->head_dim, &vs);
         if (rc != AMSKV_OK) return rc;
-        cudaError_t e = launch_append(ks, vs, cache->region(layer), lay.offset[scale], T, cache->rows, cache->heads,
-                                      cache->head_dim, (cache->flags & AMSKV_FLAG_BULK_APPEND) != 0, cache->status_word(),
-                                      cache->sm_count, static_cast<cudaStream_t>(stream));
-        if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+        Piece piece[LayerLayout::kMaxPieces];
+        const int32_t n_pieces = lay.pieces(cache->tokens, scale, piece);
+        for (int32_t i = 0; i < n_pieces; ++i) {
+            Strided kp = ks, vp = vs;
+            kp.ptr = static_cast<const __nv_bfloat16*>(ks.ptr) + (int64_t)piece[i].src * ks.token;
+            vp.ptr = static_cast<const __nv_bfloat16*>(vs.ptr) + (int64_t)piece[i].src * vs.token;
+            cudaError_t e = launch_append(kp, vp, cache->region(layer), piece[i].dst, piece[i].len, cache->rows,
+                                          cache->heads, cache->head_dim, (cache->flags & AMSKV_FLAG_BULK_APPEND) != 0,
+                                          cache->status_word(), cache->sm_count, static_cast<cudaStream_t>(stream));
+            if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+        }
     }
     const int64_t before = scale > 0 ? lay.resident_tokens(cache->tokens, scale - 1) : 0;
     const int64_t after = lay.resident_tokens(cache->tokens, scale);
@@ -398,6 +413,33 @@ int amskv_resident_ranges(const amskv_cache* cache, int layer, int scale, int32_
     for (int i = 0; i < *n; ++i) {
         ranges[2 * i] = r[i].start;
         ranges[2 * i + 1] = r[i].len;
+    }
+    return AMSKV_OK;
+}
+
+int amskv_attended_tokens(const amskv_cache* cache, int layer, int scale, int32_t* runs, int32_t* n)
+{
+    if (bad_layer_scale(cache, layer, scale) || !runs || !n) return AMSKV_ERR_INVALID;
+    TokenRun r[2 * AMSKV_MAX_SCALES];
+    *n = cache->layout[layer].attended(cache->tokens, scale, r);
+    for (int i = 0; i < *n; ++i) {
+        runs[3 * i] = r[i].segment;
+        runs[3 * i + 1] = r[i].first;
+        runs[3 * i + 2] = r[i].count;
+    }
+    return AMSKV_OK;
+}
+
+int amskv_append_copies(const amskv_cache* cache, int layer, int scale, int32_t* copies, int32_t* n)
+{
+    if (bad_layer_scale(cache, layer, scale) || !copies || !n) return AMSKV_ERR_INVALID;
+    static_assert(LayerLayout::kMaxPieces == AMSKV_MAX_APPEND_COPIES, "header and layout disagree");
+    Piece p[LayerLayout::kMaxPieces];
+    *n = cache->layout[layer].pieces(cache->tokens, scale, p);
+    for (int i = 0; i < *n; ++i) {
+        copies[3 * i] = p[i].src;
+        copies[3 * i + 1] = p[i].dst;
+        copies[3 * i + 2] = p[i].len;
     }
     return AMSKV_OK;
 }

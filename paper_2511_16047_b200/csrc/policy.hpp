@@ -14,6 +14,17 @@ struct Range {
     int32_t len;    // tokens
 };
 
+// One contiguous copy of an append: `len` tokens of the incoming scale, from its token `src`,
+// to position `dst` of the per-item region.
+struct Piece {
+    int32_t src, dst, len;
+};
+
+// `count` tokens of segment `segment`, from its token `first`.
+struct TokenRun {
+    int32_t segment, first, count;
+};
+
 // Layout of one layer.  A cache-demanding layer (or one whose pinned prefix plus window
 // already covers the whole schedule) stores its segments back to back in scale order.
 // A cache-efficient layer has a pinned region for the condensed scales and n_local slots
@@ -28,6 +39,21 @@ struct LayerLayout {
     bool full = false;      // nothing is ever evicted
     int32_t capacity = 0;   // tokens per item
     std::vector<int32_t> offset;  // [n_scales] token offset of each segment's home
+
+    // Token-budget form (Algorithm 1 with Algorithm 2 as its roll, budgets counted in tokens).
+    // The cached scales form one token stream; stream index g lives at position g while g < c_cds
+    // (the pinned head) and at c_cds + (g - c_cds) mod (c_bgt - c_cds) otherwise, so the region
+    // [0, c_bgt) is a pinned head followed by a ring whose newest tokens overwrite its oldest:
+    // exactly "the first C_cds entries and the last C_bgt - C_cds entries".  A scale that is not
+    // resident in full after its own append (larger than the budget, or larger than the ring once
+    // the ring rolls) is also written to a transient slot behind the ring, from which its own
+    // queries read it.
+    bool token_mode = false;
+    int32_t c_bgt = 0, c_cds = 0;
+    int32_t used = 0;           // positions [0, used) hold cached tokens; the transient slot starts at `used`
+    std::vector<uint8_t> cached;      // [n_scales] scale enters the stream (its size fits the budget)
+    std::vector<uint8_t> transient;   // [n_scales] scale is read from the transient slot at its own step
+    std::vector<int64_t> stream_end;  // [n_scales] stream length after the scale
 
     void build(const std::vector<int32_t>& tokens, int32_t n_condensed, int32_t n_local, bool demanding)
     {
@@ -59,7 +85,65 @@ struct LayerLayout {
         }
     }
 
-    bool keeps(int32_t s, int32_t k) const { return s <= k && (full || s < c || s > k - w); }
+    // Token-budget form: `budget` = C_bgt (C_max for a cache-demanding layer, C_min otherwise) and
+    // `condensed` = C_cds, both in tokens.  Starting a cache-demanding layer at C_max is the same as
+    // promoting it at its first overflow, because nothing is evicted before that overflow.
+    void build_tokens(const std::vector<int32_t>& tokens, int32_t budget, int32_t condensed)
+    {
+        const int32_t K = (int32_t)tokens.size();
+        token_mode = true;
+        full = false;
+        c = 0;
+        w = 1;
+        c_bgt = budget;
+        c_cds = std::min(std::max(condensed, 0), budget);
+        offset.assign(K, 0);
+        cached.assign(K, 0);
+        transient.assign(K, 0);
+        stream_end.assign(K, 0);
+        int64_t g = 0;
+        int32_t slot = 0;
+        for (int32_t s = 0; s < K; ++s) {
+            const int32_t T = tokens[s];
+            if (T <= c_bgt) {
+                cached[s] = 1;
+                const int64_t g0 = g;
+                g += T;
+                // the roll cuts into the scale itself when more of it lies behind the pinned head than the ring holds
+                const int64_t behind_head = g - std::max<int64_t>(g0, c_cds);
+                if (g > c_bgt && behind_head > c_bgt - c_cds) transient[s] = 1;
+            } else {
+                transient[s] = 1;  // never cached (Algorithm 1 skips it); attended from the transient slot
+            }
+            if (transient[s]) slot = std::max(slot, T);
+            stream_end[s] = g;
+        }
+        used = (int32_t)std::min<int64_t>(g, c_bgt);
+        capacity = used + slot;
+    }
+
+    int32_t position(int64_t g) const
+    {
+        return g < c_cds ? (int32_t)g : c_cds + (int32_t)((g - c_cds) % (c_bgt - c_cds));
+    }
+
+    // first stream index of the surviving tail after scale k (the pinned head survives besides)
+    int64_t tail_begin(int32_t k) const
+    {
+        const int64_t G = stream_end[k];
+        return G > c_bgt ? std::max<int64_t>(G - (c_bgt - c_cds), c_cds) : 0;
+    }
+
+    // does the cache hold any token of segment s right after scale k was appended
+    bool keeps(int32_t s, int32_t k) const
+    {
+        if (s > k) return false;
+        if (!token_mode) return full || s < c || s > k - w;
+        if (!cached[s]) return false;
+        const int64_t e = stream_end[s], b = s > 0 ? stream_end[s - 1] : 0;
+        if (stream_end[k] <= c_bgt) return true;
+        return b < c_cds || e > tail_begin(k);
+    }
 
     // ascending segment ids resident right after scale k was appended
     int32_t kept(int32_t k, int32_t* ids) const
@@ -70,7 +154,7 @@ struct LayerLayout {
         return n;
     }
 
-    // segments dropped by the append of scale k
+    // segments dropped by the append of scale k (a scale too large to be cached is reported at its own step)
     int32_t evicted(int32_t k, int32_t* ids) const
     {
         int32_t n = 0;
@@ -81,9 +165,51 @@ struct LayerLayout {
         return n;
     }
 
+    // the copies that append scale k; at most kMaxPieces
+    static constexpr int kMaxPieces = 4;
+    int32_t pieces(const std::vector<int32_t>& tokens, int32_t k, Piece* out) const
+    {
+        const int32_t T = tokens[k];
+        if (!token_mode) {
+            out[0] = Piece{0, offset[k], T};
+            return 1;
+        }
+        int32_t n = 0;
+        auto push = [&](int32_t src, int32_t dst, int32_t len) {
+            if (n > 0 && out[n - 1].src + out[n - 1].len == src && out[n - 1].dst + out[n - 1].len == dst) out[n - 1].len += len;
+            else out[n++] = Piece{src, dst, len};
+        };
+        if (cached[k]) {
+            const int64_t g1 = stream_end[k], g0 = g1 - T;
+            if (g0 < c_cds) push(0, (int32_t)g0, (int32_t)(std::min<int64_t>(g1, c_cds) - g0));
+            // behind the head only the tokens that survive the scale's own roll are written, so no two copies overlap
+            int64_t g = std::max<int64_t>(std::max<int64_t>(g0, c_cds), tail_begin(k));
+            while (g < g1) {
+                const int32_t p = position(g);
+                const int32_t run = (int32_t)std::min<int64_t>(g1 - g, c_bgt - p);
+                push((int32_t)(g - g0), p, run);
+                g += run;
+            }
+        }
+        if (transient[k]) push(0, used, T);
+        return n;
+    }
+
     // token ranges read at scale k, sorted by position and merged where they touch
     int32_t ranges(const std::vector<int32_t>& tokens, int32_t k, Range* out) const
     {
+        if (token_mode) {
+            int32_t n = 0;
+            int32_t res = (int32_t)std::min<int64_t>(stream_end[k], c_bgt);
+            // a scale cut by its own roll owns every resident token except the head that was there before it
+            if (transient[k] && cached[k]) res = (int32_t)std::min<int64_t>(stream_end[k] - tokens[k], c_cds);
+            if (res > 0) out[n++] = Range{0, res};
+            if (transient[k]) {
+                if (n > 0 && res == used) out[0].len += tokens[k];
+                else out[n++] = Range{used, tokens[k]};
+            }
+            return n;
+        }
         std::vector<Range> r;
         for (int32_t s = 0; s <= k; ++s)
             if (keeps(s, k)) r.push_back(Range{offset[s], tokens[s]});
@@ -96,8 +222,40 @@ struct LayerLayout {
         return n;
     }
 
+    // which tokens of which segments the queries of scale k attend to (ascending segments; at most two
+    // runs per segment: its part of the pinned head and its part of the tail)
+    int32_t attended(const std::vector<int32_t>& tokens, int32_t k, TokenRun* out) const
+    {
+        int32_t n = 0;
+        if (!token_mode) {
+            for (int32_t s = 0; s <= k; ++s)
+                if (keeps(s, k)) out[n++] = TokenRun{s, 0, tokens[s]};
+            return n;
+        }
+        const bool rolled = stream_end[k] > c_bgt;
+        const int64_t lo = tail_begin(k);
+        for (int32_t s = 0; s <= k; ++s) {
+            if (!cached[s] || (s == k && transient[k])) continue;
+            const int64_t e = stream_end[s], b = e - tokens[s];
+            if (!rolled) {
+                out[n++] = TokenRun{s, 0, tokens[s]};
+                continue;
+            }
+            const int64_t head_end = std::min<int64_t>(e, c_cds);
+            if (b < head_end) out[n++] = TokenRun{s, 0, (int32_t)(head_end - b)};
+            const int64_t t0 = std::max<int64_t>(b, lo);
+            if (t0 < e) {
+                if (n > 0 && out[n - 1].segment == s && out[n - 1].first + out[n - 1].count == t0 - b) out[n - 1].count += (int32_t)(e - t0);
+                else out[n++] = TokenRun{s, (int32_t)(t0 - b), (int32_t)(e - t0)};
+            }
+        }
+        if (transient[k]) out[n++] = TokenRun{k, 0, tokens[k]};
+        return n;
+    }
+
     int64_t resident_tokens(const std::vector<int32_t>& tokens, int32_t k) const
     {
+        if (token_mode) return std::min<int64_t>(stream_end[k], c_bgt);
         int64_t t = 0;
         for (int32_t s = 0; s <= k; ++s)
             if (keeps(s, k)) t += tokens[s];

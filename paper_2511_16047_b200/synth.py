@@ -57,6 +57,16 @@ class Workload:
         return [(self.n_condensed, self.n_local, True if full_retention else mask[i])
                 for i in range(self.layers)]
 
+    def token_budgets(self) -> List[Tuple[int, int]]:
+        """Per-layer (C_bgt, C_cds) in tokens, the way Sec. 5 sets them: C_cds = the condensed scales,
+        C_min = C_cds + the penultimate scale (cache-efficient layers), C_max = C_cds + the last two
+        scales (cache-demanding layers)."""
+        tok = self.tokens
+        cds = sum(tok[: self.n_condensed])
+        c_min = cds + (tok[-2] if len(tok) > 1 else tok[-1])
+        c_max = cds + sum(tok[-2:])
+        return [(c_max if dem else c_min, cds) for dem in self.demanding_mask()]
+
     def replace(self, **kw) -> "Workload":
         return dataclasses.replace(self, **kw)
 

@@ -29,8 +29,10 @@ def check_close(got: torch.Tensor, want: np.ndarray, what: str, max_abs=MAX_ABS,
 class Cache:
     """Thin test-side holder: creates a cache over a torch-owned arena."""
 
-    def __init__(self, layers, heads, head_dim, rows, sides, policies, softmax_scale=0.0, own_arena=True, flags=0):
-        self.desc, self._keep = B.make_desc(layers, heads, head_dim, rows, sides, policies, softmax_scale, flags)
+    def __init__(self, layers, heads, head_dim, rows, sides, policies, softmax_scale=0.0, own_arena=True, flags=0,
+                 token_budgets=None):
+        self.desc, self._keep = B.make_desc(layers, heads, head_dim, rows, sides, policies, softmax_scale, flags,
+                                            token_budgets)
         self.arena = None
         if own_arena:
             n = B.amskv_cache_required_bytes(self.desc)
