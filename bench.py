@@ -33,9 +33,9 @@ FALLBACK_BF16_TFLOPS = 1400.0
 
 # DRAM traffic of the attention kernels per step, from ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum of every attention launch of a 64-row case, scaled by rows and layers; the
-# capture is summarised under profiles/), keyed by (workload, policy).  Only valid for the
+# capture is summarised under profiles/), keyed by (workload, policy, calls).  Only valid for the
 # default batch and layer count and for the kernels as they were when it was captured.
-NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams"): 214.0e9}
+NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams", "separate"): 214.0e9}
 
 
 def _peaks():
@@ -160,8 +160,9 @@ def run_ours(args):
     outs = [torch.empty_like(q) for q, _, _ in qkv]
     input_bytes = sum(3 * q.numel() * 2 for q, _, _ in qkv)
 
-    def measure(policies, label, instrument, streams=None, budgets=None):
+    def measure(policies, label, instrument, streams=None, budgets=None, fuse=None):
         streams = args.streams if streams is None else streams
+        fuse = (args.fuse and streams == 1) if fuse is None else fuse
         desc, keep = B.make_desc(wl.layers, wl.heads, wl.head_dim, wl.rows, wl.sides, policies,
                                  flags=B.FLAG_BULK_APPEND if streams == 2 else 0, token_budgets=budgets)
         nbytes = B.amskv_cache_required_bytes(desc)
@@ -178,6 +179,8 @@ def run_ours(args):
         n_ev = wl.layers * K
         ev_app = [torch.cuda.Event() for _ in range(n_ev)] if side is not None else None
         ev_att = [torch.cuda.Event() for _ in range(n_ev)] if side is not None else None
+
+        fused_launch = {}   # (layer, scale) -> the append went into the attention launch
 
         def step(events=None):
             """Two streams: the appends run on a side stream and overlap the attention kernels of other
@@ -197,15 +200,19 @@ def run_ours(args):
                         B.amskv_append(cache, layer, k, kk, v, side)
                         ev_app[i].record(side)
                         stream.wait_event(ev_app[i])
-                    else:
+                    elif not fuse:
                         B.amskv_append(cache, layer, k, kk, v, stream)
                     if events is not None:
                         e0, e1 = events[(layer, k)]
                         e0.record(stream)
-                        B.amskv_attend(cache, layer, k, q, outs[k], stream)
-                        e1.record(stream)
+                    if fuse:
+                        n0 = B.amskv_launch_count()
+                        B.amskv_append_attend(cache, layer, k, kk, v, q, outs[k], stream)
+                        fused_launch[(layer, k)] = B.amskv_launch_count() - n0 == 1
                     else:
                         B.amskv_attend(cache, layer, k, q, outs[k], stream)
+                    if events is not None:
+                        e1.record(stream)
                     if side is not None:
                         ev_att[i].record(stream)
             if side is not None:
@@ -246,7 +253,14 @@ def run_ours(args):
             dist.barrier()
         ms = t0.elapsed_time(t1)
         result = {"label": label, "ms_per_step": ms / args.steps, "launches_per_step": launches_per_step,
-                  "kv_bytes": B.amskv_cache_bytes(cache)[2], "arena_bytes": nbytes}
+                  "kv_bytes": B.amskv_cache_bytes(cache)[2], "arena_bytes": nbytes, "fused": bool(fuse)}
+        if fuse:
+            # the timed calls now carry the append as well: the K/V of the scale written once by the fused
+            # launch (read once either way); where the call ran as two launches, also read by the copy
+            items = wl.rows * wl.heads
+            for (layer, k), (b, f) in list(work.items()):
+                kv = 2 * wl.head_dim * items * 2 * tok[k]
+                work[(layer, k)] = (b + (kv if fused_launch.get((layer, k)) else 2 * kv), f)
 
         if instrument:
             # per-launch durations of the attention kernel: same steps, eager, CUDA events on the launch stream
@@ -371,7 +385,8 @@ def run_ours(args):
         traffic = None
         if (not args.batch and not args.layers and args.path == "auto" and args.condensed is None and args.local is None
                 and args.demanding_fraction is None):
-            per_step = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy))
+            # (the capture is of the configuration named by the key; "fused" = the default calls)
+            per_step = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy, "fused" if main.get("fused") else "separate"))
             if per_step is not None:
                 traffic = round(per_step / (wl.layers * K))   # per attention launch, like `achieved`
         line = {
@@ -384,6 +399,8 @@ def run_ours(args):
                                        "x".join(map(str, wl.sides)), wl.n_condensed, wl.n_local,
                                        sum(1 for p in policies if p[2]), args.policy),
                        "step": "append + attend for every scale and layer",
+                       "calls": ("amskv_append_attend (one launch where the paired kernel takes the append in, else two)"
+                                 if main.get("fused") else "amskv_append, then amskv_attend"),
                        "l2": "inputs and per-layer KV regions far larger than L2; no flush needed",
                        "launch": "CUDA graph replay" if not args.no_graph else "eager",
                        "streams": "appends on a side stream, ordered with attention by events" if args.streams == 2 else "one stream",
@@ -391,7 +408,7 @@ def run_ours(args):
             "clocks": main["clocks"],
             "e2e": e2e,
             "gpu_launches": main["launches_per_step"] * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "attention (all attend launches of a step)",
+            "roofline": {"bound": "hbm", "kernel": "attention (all attend launches of a step; with the append fused in where amskv_append_attend does so)" if main.get("fused") else "attention (all attend launches of a step)",
                          "achieved": round(achieved, 1), "peak": hbm_gbs, "unit": "GB/s",
                          "frac": round(achieved / hbm_gbs, 4), "peak_kind": peak_kind, "traffic": traffic,
                          "algorithmic_bytes_per_launch": round(main["attend_bytes_per_step"] / (wl.layers * K)),
@@ -596,6 +613,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="var_d30")
+    ap.add_argument("--no-fuse", dest="fuse", action="store_false",
+                    help="amskv_append then amskv_attend per layer and scale instead of one amskv_append_attend call "
+                         "(the append fused into the attention launch where that pays)")
     ap.add_argument("--policy", default="ams", choices=["ams", "full", "tokens"],
                     help="ams: whole scales (condensed + local window); full: every scale; tokens: Algorithm 1 "
                          "and 2 with token budgets (C_cds = the condensed scales, C_min = C_cds + the penultimate "

@@ -175,6 +175,26 @@ AMSKV_API int amskv_append(amskv_cache* cache, int layer, int scale, const void*
 AMSKV_API int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* out,
                  const int64_t q_strides[3], const int64_t o_strides[3], void* stream);
 
+/*
+ * amskv_append(layer, scale, K, V) followed by amskv_attend(layer, scale, Q, out), with the same
+ * results, cache state and order contract (scale must be the layer's next scale), in one kernel
+ * launch where possible: Algorithm 1 appends a scale right before that scale attends, so the
+ * paired tensor-core kernel can read the scale's K and V from the caller's tensors, use them as
+ * keys and values beside the older retained tokens it reads from the cache, and write them to
+ * the scale's place in the cache on the way -- the separate copy and its second read of K and V
+ * disappear.  Scales served by the other attention kernels, appends that are more than one
+ * contiguous copy (a token budget whose ring wraps inside the scale) and, under AMSKV_PATH_AUTO,
+ * scales where splitting the current scale off its cache range would add a 64-token key tile, run
+ * as the two calls.
+ *   K, V: as for amskv_append (one stride triple kv_strides for both); Q, out: as for
+ *   amskv_attend.  out must not alias K or V.
+ * Stream ordering: as for the two calls -- this call must come after attend(layer, scale - 1)
+ * has finished reading (same stream, or an event).
+ */
+AMSKV_API int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K, const void* V,
+                                  const int64_t kv_strides[3], const void* Q, void* out, const int64_t q_strides[3],
+                                  const int64_t o_strides[3], void* stream);
+
 /* Choose the kernel used by amskv_attend (AMSKV_PATH_*).  The default is AUTO. */
 AMSKV_API int amskv_set_attend_path(amskv_cache* cache, int path);
 

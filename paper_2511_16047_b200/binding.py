@@ -60,6 +60,7 @@ def _load() -> ctypes.CDLL:
         "amskv_cache_reset": ([vp], i),
         "amskv_append": ([vp, i, i, vp, vp, i64p, vp], i),
         "amskv_attend": ([vp, i, i, vp, vp, i64p, i64p, vp], i),
+        "amskv_append_attend": ([vp, i, i, vp, vp, i64p, vp, vp, i64p, i64p, vp], i),
         "amskv_set_attend_path": ([vp, i], i),
         "amskv_step_host": ([vp, i, i, vp, vp, vp, vp, vp, sz, vp], i),
         "amskv_step_staging_bytes": ([vp, szp], i),
@@ -87,7 +88,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy amskv_cache_reset amskv_append "
-           "amskv_attend amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
+           "amskv_attend amskv_append_attend amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
            "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
            "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_attended_tokens amskv_append_copies "
            "amskv_cache_bytes amskv_status "
@@ -179,6 +180,15 @@ def amskv_append(cache: int, layer: int, scale: int, K, V, stream=None) -> None:
 def amskv_attend(cache: int, layer: int, scale: int, Q, out, stream=None) -> None:
     _check(lib.amskv_attend(cache, layer, scale, _addr(Q), _addr(out), _strides(Q), _strides(out), _stream(stream)),
            "amskv_attend")
+
+
+def amskv_append_attend(cache: int, layer: int, scale: int, K, V, Q, out, stream=None) -> None:
+    """append(layer, scale, K, V) then attend(layer, scale, Q, out), as one launch where possible."""
+    ks, vs = _strides(K), _strides(V)
+    if (ks is None) != (vs is None) or (ks is not None and list(ks) != list(vs)):
+        raise ValueError("K and V must share one stride triple")
+    _check(lib.amskv_append_attend(cache, layer, scale, _addr(K), _addr(V), ks, _addr(Q), _addr(out), _strides(Q),
+                                   _strides(out), _stream(stream)), "amskv_append_attend")
 
 
 def amskv_set_attend_path(cache: int, path: int) -> None:

@@ -136,6 +136,31 @@ int make_strided(const void* ptr, const int64_t* strides, int32_t heads, int32_t
     return AMSKV_OK;
 }
 
+// host-side state after scale `scale` of `layer` was stored
+void note_appended(amskv_cache* cache, int layer, int scale)
+{
+    const LayerLayout& lay = cache->layout[layer];
+    const int64_t before = scale > 0 ? lay.resident_tokens(cache->tokens, scale - 1) : 0;
+    const int64_t after = lay.resident_tokens(cache->tokens, scale);
+    cache->resident_now = (size_t)((int64_t)cache->resident_now + (after - before) * (int64_t)cache->token_bytes());
+    cache->peak = std::max(cache->peak, cache->resident_now);
+    cache->last_appended[layer] = scale;
+}
+
+// which kernel amskv_attend uses for T query tokens over `total` keys
+enum class AttendKernel { Small, Simt, Pair, Tensor };
+AttendKernel choose_kernel(const amskv_cache* cache, int32_t T, int32_t total)
+{
+    // AUTO: the warp-per-item kernel wherever a scale's retained keys fit its register tile, the paired
+    // tcgen05 kernel elsewhere (the CUDA-core kernel only where tensor maps are unavailable)
+    // (a single query token per item is fastest on the CUDA-core kernel: measured)
+    if ((cache->path == AMSKV_PATH_SMALL || (cache->path == AMSKV_PATH_AUTO && T > 1)) && small_supported(T, total))
+        return AttendKernel::Small;
+    if (cache->path == AMSKV_PATH_SIMT || (cache->path == AMSKV_PATH_AUTO && T == 1) || !cache->tc_ready)
+        return AttendKernel::Simt;
+    return cache->path == AMSKV_PATH_TENSOR ? AttendKernel::Tensor : AttendKernel::Pair;
+}
+
 }  // namespace
 
 extern "C" {
@@ -256,11 +281,7 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
             if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
         }
     }
-    const int64_t before = scale > 0 ? lay.resident_tokens(cache->tokens, scale - 1) : 0;
-    const int64_t after = lay.resident_tokens(cache->tokens, scale);
-    cache->resident_now = (size_t)((int64_t)cache->resident_now + (after - before) * (int64_t)cache->token_bytes());
-    cache->peak = std::max(cache->peak, cache->resident_now);
-    cache->last_appended[layer] = scale;
+    note_appended(cache, layer, scale);
     return AMSKV_OK;
 }
 
@@ -288,24 +309,17 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
     ranges.n = cache->layout[layer].ranges(cache->tokens, scale, ranges.r);
     ranges.total = 0;
     for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
-    const bool tensor = cache->path == AMSKV_PATH_TENSOR;
-    // AUTO: the warp-per-item kernel wherever a scale's retained keys fit its register tile, the paired
-    // tcgen05 kernel elsewhere (the CUDA-core kernel only where tensor maps are unavailable)
-    // (a single query token per item is fastest on the CUDA-core kernel: measured)
-    const bool small = (cache->path == AMSKV_PATH_SMALL || (cache->path == AMSKV_PATH_AUTO && T > 1)) &&
-                       small_supported(T, ranges.total);
-    const bool simt = cache->path == AMSKV_PATH_SIMT || (cache->path == AMSKV_PATH_AUTO && T == 1) || !cache->tc_ready;
-    const bool pair = !small && !simt && !tensor;
+    const AttendKernel kernel = choose_kernel(cache, T, ranges.total);
     cudaError_t e;
-    if (small) {
+    if (kernel == AttendKernel::Small) {
         e = launch_attend_small(q, o, cache->region(layer), ranges, T, cache->rows, cache->heads, cache->head_dim,
                                 cache->softmax_scale, static_cast<cudaStream_t>(stream));
-    } else if (pair) {
+    } else if (kernel == AttendKernel::Pair) {
         e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes,
                                cache->k_maps64[layer].bytes, cache->v_maps64[layer].bytes, ranges, T, cache->rows,
                                cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
                                cache->sm_count, static_cast<cudaStream_t>(stream));
-    } else if (tensor && cache->tc_ready) {
+    } else if (kernel == AttendKernel::Tensor) {
         e = launch_attend_tc(q, o, cache->region(layer), cache->k_maps[layer].bytes, cache->v_maps[layer].bytes, ranges,
                              T, cache->rows, cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
                              cache->sm_count, static_cast<cudaStream_t>(stream));
@@ -314,6 +328,67 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
                                cache->softmax_scale, static_cast<cudaStream_t>(stream));
     }
     if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
+}
+
+int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K, const void* V,
+                        const int64_t kv_strides[3], const void* Q, void* out, const int64_t q_strides[3],
+                        const int64_t o_strides[3], void* stream)
+{
+    if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
+    if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
+    const int32_t T = cache->tokens[scale];
+    const LayerLayout& lay = cache->layout[layer];
+    Strided ks, vs, q, o;
+    int rc = make_strided(K, kv_strides, cache->heads, T, cache->head_dim, &ks);
+    if (rc == AMSKV_OK) rc = make_strided(V, kv_strides, cache->heads, T, cache->head_dim, &vs);
+    if (rc == AMSKV_OK) rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
+    if (rc == AMSKV_OK) rc = make_strided(out, o_strides, cache->heads, T, cache->head_dim, &o);
+    if (rc != AMSKV_OK) return rc;
+    // One launch where the paired kernel serves this scale and the append is a single copy: the kernel
+    // reads the scale from K and V, attends to it together with the older retained tokens, and writes
+    // it to its place in the cache on the way.  Elsewhere: the two calls, one after the other.
+    RangeList after;
+    after.n = lay.ranges(cache->tokens, scale, after.r);
+    after.total = 0;
+    for (int i = 0; i < after.n; ++i) after.total += after.r[i].len;
+    Piece piece[LayerLayout::kMaxPieces];
+    const int32_t n_pieces = lay.pieces(cache->tokens, scale, piece);
+    bool fused = cache->tc_ready && choose_kernel(cache, T, after.total) == AttendKernel::Pair && n_pieces == 1 &&
+                 piece[0].src == 0 && piece[0].len == T;
+    RangeList ranges;
+    if (fused) {
+        ranges.n = lay.ranges_before(cache->tokens, scale, ranges.r);
+        if (ranges.n >= kMaxRanges) fused = false;
+    }
+    if (fused && cache->path == AMSKV_PATH_AUTO) {
+        // The kernel works in 64-token key tiles per range.  Taking the scale from the caller's tensors
+        // splits it off the range it would be part of in the cache; where that adds a tile, attention
+        // loses more than the saved copy is worth (measured), so such scales run as the two calls
+        // (AMSKV_PATH_TENSOR_PAIR fuses wherever it can).
+        auto tiles = [](const RangeList& rl) {
+            int32_t n = 0;
+            for (int i = 0; i < rl.n; ++i) n += (rl.r[i].len + 63) / 64;
+            return n;
+        };
+        if (tiles(ranges) + (T + 63) / 64 > tiles(after)) fused = false;
+    }
+    if (!fused) {
+        rc = amskv_append(cache, layer, scale, K, V, kv_strides, stream);
+        if (rc != AMSKV_OK) return rc;
+        return amskv_attend(cache, layer, scale, Q, out, q_strides, o_strides, stream);
+    }
+    ranges.r[ranges.n++] = Range{0, T};   // the current scale, in the caller's tensors
+    ranges.total = 0;
+    for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
+    CurrentScaleSource cur{ks, vs, true, piece[0].dst, cache->region(layer)};
+    cudaError_t e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes,
+                                       cache->k_maps64[layer].bytes, cache->v_maps64[layer].bytes, ranges, T, cache->rows,
+                                       cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),
+                                       cache->sm_count, static_cast<cudaStream_t>(stream), &cur);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    note_appended(cache, layer, scale);
     return AMSKV_OK;
 }
 
@@ -345,9 +420,7 @@ int amskv_step_host(amskv_cache* cache, int layer, int scale, const void* K_host
     if (e == cudaSuccess) e = cudaMemcpyAsync(s + one, V_host, bytes, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(s + 2 * one, Q_host, bytes, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
-    int rc = amskv_append(cache, layer, scale, s, s + one, nullptr, stream);
-    if (rc != AMSKV_OK) return rc;
-    rc = amskv_attend(cache, layer, scale, s + 2 * one, s + 3 * one, nullptr, nullptr, stream);
+    int rc = amskv_append_attend(cache, layer, scale, s, s + one, nullptr, s + 2 * one, s + 3 * one, nullptr, nullptr, stream);
     if (rc != AMSKV_OK) return rc;
     e = cudaMemcpyAsync(out_host, s + 3 * one, bytes, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }

@@ -82,6 +82,19 @@ struct PairPlan {
     int32_t n_pairs;
 };
 
+// The current scale read from the caller's K/V tensors instead of the cache: the last entry of the
+// range list stands for it (start 0, len T).  With `store` every tile fetched that way is also written
+// to the scale's place in the cache (the append fused into attention).
+constexpr int32_t kExtFlag = 1 << 30;   // marks such a tile's first token in the tile table
+struct ExtArgs {
+    CUtensorMap k64, v64, k16, v16;   // rank-4 maps of the caller's K and V (64- and 16-token boxes)
+    CUtensorMap k_store, v_store;     // the layer's region, clipped at the end of the scale's place (64-token boxes)
+    int32_t range;                    // index of the range that stands for the current scale
+    int32_t store;
+    int32_t dst;                      // first position of the scale in the per-item region
+    int3 pos;                         // coordinate slots of token, head and row in the rank-4 maps
+};
+
 struct Stream {
     int32_t item;
     int32_t qt;
@@ -173,6 +186,17 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // True in exactly one lane of a converged warp.
 __device__ __forceinline__ bool elect_one()
@@ -379,7 +403,8 @@ __device__ __forceinline__ void report(int* status, int code, volatile int* abor
 }
 
 // Tile j of the resident ranges: first token and number of valid tokens (<= 64).
-__device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0, int32_t& valid)
+// A tile of range `ext_range` (the current scale in the caller's tensors) carries kExtFlag in t0.
+__device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0, int32_t& valid, int ext_range = -1)
 {
     int r = 0;
     for (; r < rl.n - 1; ++r) {
@@ -389,17 +414,20 @@ __device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0,
     }
     t0 = rl.r[r].start + j * kKT;
     valid = min(kKT, rl.r[r].start + rl.r[r].len - t0);
+    if (r == ext_range) t0 |= kExtFlag;
 }
 
 // ---------------------------------------------------------------- kernel
-template <int D>
+template <int D, bool kExt>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::kCtasPerSm)
 attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap k_map64,
-                   const __grid_constant__ CUtensorMap v_map64, __nv_bfloat16* __restrict__ O, int64_t o_row,
+                   const __grid_constant__ CUtensorMap v_map64, const __grid_constant__ ExtArgs ext,
+                   __nv_bfloat16* __restrict__ O, int64_t o_row,
                    int64_t o_head, int64_t o_tok, const RangeList ranges, int32_t T, int32_t heads,
                    const PairPlan pp, int32_t n_tiles, int3 qpos, float scale_log2, int* __restrict__ status)
 {
+    const int ext_range = kExt ? ext.range : -1;
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     Barriers* bars = reinterpret_cast<Barriers*>(smem_raw);
@@ -431,7 +459,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
     for (int j = threadIdx.x; j < n_tiles && j < kTileTab; j += kThreads) {
         int32_t t0, valid;
-        tile_at(ranges, j, t0, valid);
+        tile_at(ranges, j, t0, valid, ext_range);
         bars->tile_tab[j] = make_int2(t0, valid);
     }
     if (layout_ok) {
@@ -456,7 +484,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             t0 = e.x;
             valid = e.y;
         } else {
-            tile_at(ranges, j, t0, valid);
+            tile_at(ranges, j, t0, valid, ext_range);
         }
     };
 
@@ -480,17 +508,56 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         // ------------------------------------------------------------ TMA producer of K/V tiles
         uint32_t sq = 0;  // stages issued so far
         bool ok = true;
+        // Fused append: a tile of the current scale is written to the cache two stages after it was
+        // requested (it has landed by then, so the wait costs nothing), by lane 0, as one bulk group per
+        // stage; before a stage is refilled, every group but the two newest has finished reading it.
+        const bool storing = kExt && ext.store != 0;
+        uint32_t st_sq[2] = {0, 0};
+        int32_t st_tok[2] = {0, 0}, st_item[2] = {0, 0};
+        int st_n = 0;
+        auto store_front = [&]() -> bool {
+            const uint32_t stage = st_sq[0] % C::kStages, use = st_sq[0] / C::kStages;
+            if (!warp_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) return false;
+            if (lane == 0) {
+                const uint32_t k_src = kv_smem + stage * C::kStageBytes, v_src = k_src + C::kKVBytes;
+#pragma unroll
+                for (int h = 0; h < C::kHalves; ++h) {
+                    tma_store_3d(&ext.k_store, k_src + h * C::kKVHalfBytes, h * 64, ext.dst + st_tok[0], st_item[0]);
+                    tma_store_3d(&ext.v_store, v_src + h * C::kKVHalfBytes, h * 64, ext.dst + st_tok[0], st_item[0]);
+                }
+            }
+            st_sq[0] = st_sq[1];
+            st_tok[0] = st_tok[1];
+            st_item[0] = st_item[1];
+            --st_n;
+            return true;
+        };
         for (uint32_t n = 0; ok && n < my_pairs; ++n) {
             const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
             const Stream sa = stream_of(pp, pair, 0), sb = stream_of(pp, pair, 1);
             const int per_tile = (!pp.two_q && sb.valid) ? 2 : 1;
+            // one unit per item writes the item's tiles: with two query tiles per unit, the unit of the first tiles
+            const bool unit_stores = storing && (!pp.two_q || sa.qt == 0);
             for (int j = 0; ok && j < n_tiles; ++j) {
                 int32_t t0, valid;
                 tile_of(j, t0, valid);
+                const bool from_ext = kExt && (t0 & kExtFlag) != 0;
+                t0 &= ~kExtFlag;
                 const int nch = (valid + 15) >> 4;
                 for (int g = 0; g < per_tile; ++g, ++sq) {
                     const int item = g == 0 ? sa.item : sb.item;
                     const uint32_t stage = sq % C::kStages, use = sq / C::kStages;
+                    if (storing) {
+                        if (st_n > 0 && st_sq[0] + 2 <= sq && !store_front()) {
+                            ok = false;
+                            break;
+                        }
+                        if (lane == 0) {
+                            bulk_commit();
+                            bulk_wait_read<2>();
+                        }
+                        __syncwarp();
+                    }
                     if (!warp_wait(kv_empty0 + 8 * stage, (use & 1u) ^ 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -499,7 +566,31 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     const uint32_t k_dst = kv_smem + stage * C::kStageBytes, v_dst = k_dst + C::kKVBytes;
                     if (elect_one()) {
                         mbar_expect_tx(full, (uint32_t)nch * kKVBoxRows * D * 2 * 2);
-                        if (nch == kKT / kKVBoxRows) {
+                        if (from_ext) {
+                            const int32_t row = item / heads, head = item - row * heads;
+                            int c[4] = {0, 0, 0, 0};
+                            c[ext.pos.y] = head;
+                            c[ext.pos.z] = row;
+                            if (nch == kKT / kKVBoxRows) {
+                                c[ext.pos.x] = t0;
+#pragma unroll
+                                for (int h = 0; h < C::kHalves; ++h) {
+                                    tma_load_4d(k_dst + h * C::kKVHalfBytes, &ext.k64, full, h * 64, c[1], c[2], c[3]);
+                                    tma_load_4d(v_dst + h * C::kKVHalfBytes, &ext.v64, full, h * 64, c[1], c[2], c[3]);
+                                }
+                            } else {
+                                for (int bx = 0; bx < nch; ++bx) {
+                                    c[ext.pos.x] = t0 + bx * kKVBoxRows;
+#pragma unroll
+                                    for (int h = 0; h < C::kHalves; ++h) {
+                                        tma_load_4d(k_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &ext.k16, full, h * 64,
+                                                    c[1], c[2], c[3]);
+                                        tma_load_4d(v_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &ext.v16, full, h * 64,
+                                                    c[1], c[2], c[3]);
+                                    }
+                                }
+                            }
+                        } else if (nch == kKT / kKVBoxRows) {
 #pragma unroll
                             for (int h = 0; h < C::kHalves; ++h) {
                                 tma_load_3d(k_dst + h * C::kKVHalfBytes, &k_map64, full, h * 64, t0, item);
@@ -518,8 +609,22 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         }
                     }
                     __syncwarp();
+                    if (from_ext && unit_stores) {
+                        st_sq[st_n] = sq;
+                        st_tok[st_n] = t0;
+                        st_item[st_n] = item;
+                        ++st_n;
+                    }
                 }
             }
+        }
+        if (storing) {
+            while (ok && st_n > 0) ok = store_front();
+            if (lane == 0) {
+                bulk_commit();
+                bulk_wait_all();   // the writes are complete, and the stages no longer read, before the CTA ends
+            }
+            __syncwarp();
         }
         if (!ok) {
             if (lane == 0) report(status, kStatusTmaTimeout, abort_flag);
@@ -837,25 +942,25 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 }
 
 // ---------------------------------------------------------------- host side
-template <int D>
+template <int D, bool kExt>
 cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& km64,
-                   const CUtensorMap& vm64, const Strided& O,
+                   const CUtensorMap& vm64, const ExtArgs& ext, const Strided& O,
                    const RangeList& ranges, int32_t T, int32_t heads, const PairPlan& pp, int32_t n_tiles, int3 qpos,
                    float scale_log2, int* status, int sm_count, cudaStream_t stream)
 {
     using C = Cfg<D>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attend_pair_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(attend_pair_kernel<D, kExt>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)C::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > pp.n_pairs) grid = pp.n_pairs;
-    attend_pair_kernel<D><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(
-        qm, km, vm, km64, vm64, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos, scale_log2,
-        status);
+    attend_pair_kernel<D, kExt><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(
+        qm, km, vm, km64, vm64, ext, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos,
+        scale_log2, status);
     count_launch();
     return cudaGetLastError();
 }
@@ -864,9 +969,31 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
 
 cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map, const void* v_map,
                                const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
-                               float softmax_scale, int* status, int sm_count, cudaStream_t stream)
+                               float softmax_scale, int* status, int sm_count, cudaStream_t stream,
+                               const CurrentScaleSource* cur)
 {
     if (ranges.n < 1 || ranges.total < 1 || T < 1) return cudaErrorInvalidValue;
+    ExtArgs ext;
+    memset(&ext, 0, sizeof(ext));
+    ext.range = -1;
+    if (cur) {
+        // the last range stands for the current scale, whose tokens come from the caller's tensors
+        if (ranges.r[ranges.n - 1].start != 0 || ranges.r[ranges.n - 1].len != T) return cudaErrorInvalidValue;
+        int kp[3], vp[3];
+        if (!tc_encode_q_map(cur->K, T, rows, heads, D, kKT, &ext.k64, kp) ||
+            !tc_encode_q_map(cur->V, T, rows, heads, D, kKT, &ext.v64, vp) ||
+            !tc_encode_q_map(cur->K, T, rows, heads, D, kKVBoxRows, &ext.k16, kp) ||
+            !tc_encode_q_map(cur->V, T, rows, heads, D, kKVBoxRows, &ext.v16, vp))
+            return cudaErrorNotSupported;
+        if (kp[0] != vp[0] || kp[1] != vp[1] || kp[2] != vp[2]) return cudaErrorNotSupported;
+        ext.pos = make_int3(kp[0], kp[1], kp[2]);
+        ext.range = ranges.n - 1;
+        ext.store = cur->store ? 1 : 0;
+        ext.dst = cur->dst;
+        if (cur->store &&
+            !tc_encode_kv_store_maps(cur->region, (int64_t)rows * heads, D, kKT, cur->dst + T, &ext.k_store, &ext.v_store))
+            return cudaErrorNotSupported;
+    }
     CUtensorMap qm;
     int pos[3];
     if (!tc_encode_q_map(Q, T, rows, heads, D, kQBoxRows, &qm, pos)) return cudaErrorNotSupported;
@@ -886,9 +1013,18 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     for (int i = 0; i < ranges.n; ++i) n_tiles += (ranges.r[i].len + kKT - 1) / kKT;
     const int3 qpos = make_int3(pos[0], pos[1], pos[2]);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
+    if (cur) {
+        if (D == 64)
+            return launch<64, true>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
+                                    sm_count, stream);
+        return launch<128, true>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
+                                 sm_count, stream);
+    }
     if (D == 64)
-        return launch<64>(qm, km, vm, km64, vm64, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status, sm_count, stream);
-    return launch<128>(qm, km, vm, km64, vm64, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status, sm_count, stream);
+        return launch<64, false>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
+                                 sm_count, stream);
+    return launch<128, false>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
+                              sm_count, stream);
 }
 
 }  // namespace amskv

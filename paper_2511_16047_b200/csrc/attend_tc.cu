@@ -600,6 +600,21 @@ bool tc_encode_kv_maps(const LayerRegion& region, int64_t items, int32_t D, int 
     return true;
 }
 
+bool tc_encode_kv_store_maps(const LayerRegion& region, int64_t items, int32_t D, int box_rows, int32_t token_extent,
+                             void* k_map_out, void* v_map_out)
+{
+    if (token_extent < 1 || token_extent > region.capacity) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)token_extent, (cuuint64_t)items};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)region.capacity * D * 2 * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    CUtensorMap km, vm;
+    if (!encode_map(&km, region.base, 3, dims, strides, box)) return false;
+    if (!encode_map(&vm, region.base + (int64_t)region.capacity * D, 3, dims, strides, box)) return false;
+    memcpy(k_map_out, &km, sizeof(km));
+    memcpy(v_map_out, &vm, sizeof(vm));
+    return true;
+}
+
 // Q as a rank-4 tensor: channels, then token / head / row ordered by ascending stride.  pos[0..2]
 // receive the coordinate index (1..3) of the token, head and row dimensions.
 bool tc_encode_q_map(const Strided& Q, int32_t T, int32_t rows, int32_t heads, int32_t D, int box_rows, void* map_out,

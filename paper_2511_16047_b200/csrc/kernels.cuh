@@ -68,10 +68,26 @@ cudaError_t launch_attend_tc(const Strided& Q, const Strided& O, const LayerRegi
 // Encodes the rank-4 tensor map of a strided Q tensor (box = 64 channels x box_rows tokens).
 bool tc_encode_q_map(const Strided& Q, int32_t T, int32_t rows, int32_t heads, int32_t D, int box_rows, void* map_out,
                      int pos[3]);
+// The layer's region as store targets (box = 64 channels x box_rows tokens) whose token extent ends at
+// `token_extent`, so that a box reaching past it is clipped by the copy engine.
+bool tc_encode_kv_store_maps(const LayerRegion& region, int64_t items, int32_t D, int box_rows, int32_t token_extent,
+                             void* k_map_out, void* v_map_out);
+
+// The current scale taken from the caller's K/V tensors instead of the cache: the last entry of the
+// range list given with it stands for that scale (start 0, len T).  With `store`, the kernel also
+// writes the scale to position `dst` of every item's part of `region` (the append fused into attention).
+struct CurrentScaleSource {
+    Strided K, V;
+    bool store;
+    int32_t dst;
+    LayerRegion region;
+};
+
 // Paired tensor-core kernel: two softmax groups per CTA, probabilities kept in tensor memory.
 cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map16, const void* v_map16,
                                const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
-                               float softmax_scale, int* status, int sm_count, cudaStream_t stream);
+                               float softmax_scale, int* status, int sm_count, cudaStream_t stream,
+                               const CurrentScaleSource* cur = nullptr);
 
 // Warp-per-item kernel for the coarse scales: every retained key in one register tile.
 constexpr int kSmallMaxKeys = 32;

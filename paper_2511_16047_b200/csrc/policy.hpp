@@ -253,6 +253,40 @@ struct LayerLayout {
         return n;
     }
 
+    // token ranges of the segments other than k that the queries of scale k attend to (sorted, merged):
+    // what attention reads from the cache when scale k itself comes from the caller's tensors.  These
+    // positions are not touched by the append of scale k, so they may be read while it is written.
+    int32_t ranges_before(const std::vector<int32_t>& tokens, int32_t k, Range* out) const
+    {
+        TokenRun runs[2 * 32];
+        const int32_t n_runs = attended(tokens, k, runs);
+        std::vector<Range> r;
+        for (int32_t i = 0; i < n_runs; ++i) {
+            const int32_t s = runs[i].segment;
+            if (s == k) continue;
+            if (!token_mode) {
+                r.push_back(Range{offset[s] + runs[i].first, runs[i].count});
+                continue;
+            }
+            int64_t g = (s > 0 ? stream_end[s - 1] : 0) + runs[i].first;
+            int32_t left = runs[i].count;
+            while (left > 0) {
+                const int32_t p = g < c_cds ? (int32_t)g : position(g);
+                const int32_t run = std::min<int32_t>(left, (g < c_cds ? c_cds : c_bgt) - p);
+                r.push_back(Range{p, run});
+                g += run;
+                left -= run;
+            }
+        }
+        std::sort(r.begin(), r.end(), [](const Range& a, const Range& b) { return a.start < b.start; });
+        int32_t n = 0;
+        for (const Range& x : r) {
+            if (n > 0 && out[n - 1].start + out[n - 1].len == x.start) out[n - 1].len += x.len;
+            else out[n++] = x;
+        }
+        return n;
+    }
+
     int64_t resident_tokens(const std::vector<int32_t>& tokens, int32_t k) const
     {
         if (token_mode) return std::min<int64_t>(stream_end[k], c_bgt);

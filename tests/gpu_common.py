@@ -63,17 +63,21 @@ def tensor_path_available(head_dim=64) -> bool:
         return B.lib.amskv_set_attend_path(c.h, B.PATH_TENSOR) == B.OK
 
 
-def run_pass(cache: Cache, qkv, path=B.PATH_AUTO, layers=None):
-    """Appends and attends every scale; qkv[k] = (Q, K, V) device tensors.  Returns outs[layer][k]."""
+def run_pass(cache: Cache, qkv, path=B.PATH_AUTO, layers=None, fused=False):
+    """Appends and attends every scale; qkv[k] = (Q, K, V) device tensors.  Returns outs[layer][k].
+    fused: through amskv_append_attend (True), or only at the scales listed."""
     B.amskv_cache_reset(cache.h)
     B.amskv_set_attend_path(cache.h, path)
     layers = range(len(cache.policies)) if layers is None else layers
     outs = {l: [] for l in layers}
     for k, (q, kk, v) in enumerate(qkv):
         for l in layers:
-            B.amskv_append(cache.h, l, k, kk, v)
             o = torch.full_like(q, float("nan"))
-            B.amskv_attend(cache.h, l, k, q, o)
+            if fused is True or (fused and k in fused):
+                B.amskv_append_attend(cache.h, l, k, kk, v, q, o)
+            else:
+                B.amskv_append(cache.h, l, k, kk, v)
+                B.amskv_attend(cache.h, l, k, q, o)
             outs[l].append(o)
     torch.cuda.synchronize()
     assert B.amskv_status(cache.h) == 0
