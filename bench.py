@@ -31,11 +31,11 @@ UNIT = "us/image"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0
 
-# DRAM traffic of the attention kernels per step, from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of every attention launch of a 64-row case, scaled by rows and layers; the
+# DRAM traffic of the timed calls per step, from ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum of every launch of those calls in a 64-row case, scaled by rows and layers; the
 # capture is summarised under profiles/), keyed by (workload, policy, calls).  Only valid for the
 # default batch and layer count and for the kernels as they were when it was captured.
-NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams", "separate"): 214.0e9}
+NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams", "fused"): 278.7e9}
 
 
 def _peaks():
