@@ -51,6 +51,19 @@ def test_large_problem_uses_grid_stride_and_fixed_partials():
     assert abs(got - want) <= 1e-5 * want
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_few_items_with_long_sides_are_split_into_parts(D):
+    """Two items of 48 x 48 tokens: each item is cut into many block-sized parts (with a ragged last one);
+    also a larger previous scale than current one (downsampling), which the bilinear rule covers as well."""
+    rows, heads = 1, 2
+    kp = synth.normal_bf16((rows, heads, 40 * 40, D), 7, "cuda")
+    kc = synth.normal_bf16((rows, heads, 48 * 48, D), 8, "cuda")
+    for a, sa, b, sb in ((kp, 40, kc, 48), (kc, 48, kp, 40)):
+        got = _gpu_ss(a, sa, b, sb, rows, heads, D)
+        want = oracle.similarity_ss(to_items(a), sa, to_items(b), sb)
+        assert abs(got - want) <= 1e-5 * want
+
+
 def test_correlated_layers_rank_above_independent_ones():
     rows, heads, D = 4, 8, 64
     sides = (4, 5, 6, 8, 10)
