@@ -417,7 +417,7 @@ def run_ours(args):
             "pass_roofline": {"roofline_ms": round(main["pass_roofline_ms"], 3),
                               "attend_ms": round(main["attend_ms_per_step"], 3),
                               "frac": round(main["pass_roofline_ms"] / main["attend_ms_per_step"], 4),
-                              "note": "sum over launches of max(bytes/HBM peak, flops/bf16 peak) / measured attention time"},
+                              "note": "sum over the timed calls of max(bytes/HBM peak, flops/bf16 peak) / their measured time"},
             "attend_only_us_per_image": round(main["attend_ms_per_step"] * 1e3 / wl.batch, 3),
             "eager_ms_per_step": round(main["eager_ms_per_step"], 4),
             "kv_cache_gb": round(main["kv_bytes"] / 1e9, 3),
