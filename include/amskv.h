@@ -58,7 +58,8 @@ extern "C" {
 
 /* amskv_desc.flags */
 #define AMSKV_FLAG_PLAN_ONLY 1u /* host bookkeeping only: no device memory is touched and
-                                   attend / similarity are refused; append takes NULL K, V.
+                                   attend / similarity are refused; append takes NULL K, V
+                                   (append_attend does the bookkeeping of append, whatever its pointers).
                                    For sizing and for inspecting the policy without a GPU. */
 
 #define AMSKV_FLAG_BULK_APPEND 2u /* amskv_append moves token-contiguous inputs with bulk asynchronous
@@ -67,6 +68,17 @@ extern "C" {
                                     kernel's CTAs.  Meant for callers that enqueue appends on a side
                                     stream underneath attention; on its own it is a little slower
                                     than the default copy kernel. */
+
+#define AMSKV_FLAG_TRANSIENT_LAST_SCALE 4u /* The last scale of the schedule is never stored: no later scale
+                                    reads it (Algorithm 1 would append it all the same).  The arena reserves no
+                                    room for it -- a cache-demanding layer of the 680-token schedule holds 424
+                                    tokens instead of 680, a cache-efficient one (2 condensed, 2 local scales) 274
+                                    instead of 430 -- and its step must be made through amskv_append_attend
+                                    (or amskv_step_host), which reads the scale's K and V from the caller's
+                                    tensors; amskv_append refuses it with AMSKV_ERR_UNSUPPORTED.  The attention
+                                    result is the same as without the flag.  The policy queries report the
+                                    scale as not retained (amskv_kept_segments) and as dropped at its own step
+                                    (amskv_evicted_at). */
 
 /* amskv_set_attend_path */
 #define AMSKV_PATH_AUTO 0   /* CUDA-core kernel for a single query token, warp-per-item kernel for the

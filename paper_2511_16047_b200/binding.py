@@ -20,6 +20,7 @@ ERR_INVALID, ERR_ORDER, ERR_NOMEM, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT
 MAX_SCALES = 32
 FLAG_PLAN_ONLY = 1
 FLAG_BULK_APPEND = 2
+FLAG_TRANSIENT_LAST_SCALE = 4
 PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_PAIR, PATH_SMALL = 0, 1, 2, 3, 4
 
 

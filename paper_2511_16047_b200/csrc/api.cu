@@ -46,6 +46,8 @@ struct amskv_cache {
     size_t resident_now = 0, peak = 0;
 
     bool plan_only() const { return (flags & AMSKV_FLAG_PLAN_ONLY) != 0; }
+    // the scale is the last one of a cache that never stores its last scale
+    bool transient(int scale) const { return (flags & AMSKV_FLAG_TRANSIENT_LAST_SCALE) != 0 && scale == n_scales - 1; }
     int64_t items() const { return (int64_t)rows * heads; }
     size_t token_bytes() const { return (size_t)items() * head_dim * 2 /*bf16*/ * 2 /*K and V*/; }
     LayerRegion region(int layer) const
@@ -72,7 +74,8 @@ int check_desc(const amskv_desc* d)
         }
         if (d->policy[l].n_condensed < 0 || d->policy[l].n_local < 1) return AMSKV_ERR_INVALID;
     }
-    if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND)) != 0) return AMSKV_ERR_INVALID;
+    if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND | AMSKV_FLAG_TRANSIENT_LAST_SCALE)) != 0)
+        return AMSKV_ERR_INVALID;
     if (!(d->softmax_scale == d->softmax_scale)) return AMSKV_ERR_INVALID;  // NaN
     return AMSKV_OK;
 }
@@ -98,10 +101,13 @@ int plan(const amskv_desc* d, amskv_cache* c)
     c->layer_offset.resize(d->layers);
     size_t at = kStatusBytes;
     for (int l = 0; l < d->layers; ++l) {
+        const bool transient_last = (d->flags & AMSKV_FLAG_TRANSIENT_LAST_SCALE) != 0;
         if (d->token_budget && d->token_budget[l].budget_tokens > 0)
-            c->layout[l].build_tokens(c->tokens, d->token_budget[l].budget_tokens, d->token_budget[l].condensed_tokens);
+            c->layout[l].build_tokens(c->tokens, d->token_budget[l].budget_tokens, d->token_budget[l].condensed_tokens,
+                                      transient_last);
         else
-            c->layout[l].build(c->tokens, d->policy[l].n_condensed, d->policy[l].n_local, d->policy[l].cache_demanding != 0);
+            c->layout[l].build(c->tokens, d->policy[l].n_condensed, d->policy[l].n_local,
+                               d->policy[l].cache_demanding != 0, transient_last);
         if ((int64_t)c->layout[l].capacity > (1ll << 30)) return AMSKV_ERR_INVALID;
         c->layer_offset[l] = at;
         at += align_up((size_t)c->layout[l].capacity * c->token_bytes());
@@ -261,6 +267,7 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
 {
     if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
     if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
+    if (cache->transient(scale)) return AMSKV_ERR_UNSUPPORTED;   // it has no place in the arena: amskv_append_attend
     const int32_t T = cache->tokens[scale];
     const LayerLayout& lay = cache->layout[layer];
     if (!cache->plan_only()) {
@@ -336,8 +343,11 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
                         const int64_t o_strides[3], void* stream)
 {
     if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
-    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
     if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
+    if (cache->plan_only()) {   // bookkeeping only
+        note_appended(cache, layer, scale);
+        return AMSKV_OK;
+    }
     const int32_t T = cache->tokens[scale];
     const LayerLayout& lay = cache->layout[layer];
     Strided ks, vs, q, o;
@@ -346,6 +356,29 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
     if (rc == AMSKV_OK) rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
     if (rc == AMSKV_OK) rc = make_strided(out, o_strides, cache->heads, T, cache->head_dim, &o);
     if (rc != AMSKV_OK) return rc;
+    if (cache->transient(scale)) {
+        // Never stored: the queries attend to the older retained tokens in the cache and to the scale's own
+        // K and V straight from the caller's tensors (paired kernel, else the CUDA-core kernel).
+        RangeList rl;
+        rl.n = lay.ranges_before(cache->tokens, scale, rl.r);
+        if (rl.n >= kMaxRanges) return AMSKV_ERR_UNSUPPORTED;
+        rl.r[rl.n++] = Range{0, T};
+        rl.total = 0;
+        for (int i = 0; i < rl.n; ++i) rl.total += rl.r[i].len;
+        CurrentScaleSource src{ks, vs, false, 0, cache->region(layer)};
+        cudaError_t e;
+        if (cache->tc_ready && cache->path != AMSKV_PATH_SIMT && !(cache->path == AMSKV_PATH_AUTO && T == 1))
+            e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes, cache->k_maps64[layer].bytes,
+                                   cache->v_maps64[layer].bytes, rl, T, cache->rows, cache->heads, cache->head_dim,
+                                   cache->softmax_scale, cache->status_word(), cache->sm_count,
+                                   static_cast<cudaStream_t>(stream), &src);
+        else
+            e = launch_attend_simt(q, o, cache->region(layer), rl, T, cache->rows, cache->heads, cache->head_dim,
+                                   cache->softmax_scale, static_cast<cudaStream_t>(stream), &src);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+        note_appended(cache, layer, scale);
+        return AMSKV_OK;
+    }
     // One launch where the paired kernel serves this scale and the append is a single copy: the kernel
     // reads the scale from K and V, attends to it together with the older retained tokens, and writes
     // it to its place in the cache on the way.  Elsewhere: the two calls, one after the other.

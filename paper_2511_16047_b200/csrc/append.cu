@@ -174,12 +174,9 @@ cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion&
     const bool contiguous = K.token == D && V.token == D && K.head == (int64_t)T * D && V.head == (int64_t)T * D &&
                             K.row == (int64_t)heads * T * D && V.row == (int64_t)heads * T * D;
     if (bulk && contiguous && block_bytes >= 4096 && block_bytes < (1ll << 31)) {
-        static bool configured = false;
-        if (!configured) {
-            cudaError_t e = cudaFuncSetAttribute(append_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmem);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
+        static SharedMemoryOptIn opt_in;
+        const cudaError_t oe = opt_in.ensure(append_bulk_kernel, (int)kBulkSmem);
+        if (oe != cudaSuccess) return oe;
         const uint32_t cpb = (uint32_t)((block_bytes + kBulkChunk - 1) / kBulkChunk);
         const int64_t total_chunks = (int64_t)rows * heads * 2 * cpb;
         int64_t grid = (int64_t)(sm_count > 0 ? sm_count : 148) * 8;

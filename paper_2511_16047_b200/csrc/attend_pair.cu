@@ -949,13 +949,9 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
                    float scale_log2, int* status, int sm_count, cudaStream_t stream)
 {
     using C = Cfg<D>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attend_pair_kernel<D, kExt>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static SharedMemoryOptIn opt_in;
+    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt>, (int)C::kSmemBytes);
+    if (oe != cudaSuccess) return oe;
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > pp.n_pairs) grid = pp.n_pairs;
     attend_pair_kernel<D, kExt><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(

@@ -46,7 +46,8 @@ __global__ void __launch_bounds__(kThreads)
 attend_simt_kernel(const __nv_bfloat16* __restrict__ Q, int64_t q_row, int64_t q_head, int64_t q_tok,
                    __nv_bfloat16* __restrict__ O, int64_t o_row, int64_t o_head, int64_t o_tok,
                    const __nv_bfloat16* __restrict__ region, int32_t capacity, const RangeList ranges, int32_t T,
-                   int32_t heads, int64_t total_rows, float scale_log2)
+                   int32_t heads, int64_t total_rows, float scale_log2, const __nv_bfloat16* __restrict__ ext_k,
+                   const __nv_bfloat16* __restrict__ ext_v, int64_t e_row, int64_t e_head, int64_t e_tok, int ext_range)
 {
     constexpr int DPL = D / kLanesPerRow;  // channels per lane
     const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -73,6 +74,11 @@ attend_simt_kernel(const __nv_bfloat16* __restrict__ Q, int64_t q_row, int64_t q
     for (int d = 0; d < DPL; ++d) o[d] = 0.f;
 
     for (int r = 0; r < ranges.n; ++r) {
+        // range `ext_range` (if any) is the current scale in the caller's own K and V tensors
+        const bool ext = r == ext_range;
+        const __nv_bfloat16* kb = ext ? ext_k + row * e_row + head * e_head + sub * DPL : kbase;
+        const __nv_bfloat16* vb = ext ? ext_v + row * e_row + head * e_head + sub * DPL : vbase;
+        const int64_t tstride = ext ? e_tok : (int64_t)D;
         const int32_t end = ranges.r[r].start + ranges.r[r].len;
         for (int32_t tok = ranges.r[r].start; tok < end; tok += kKeysPerStep) {
             float s[kKeysPerStep];
@@ -81,8 +87,8 @@ attend_simt_kernel(const __nv_bfloat16* __restrict__ Q, int64_t q_row, int64_t q
             for (int u = 0; u < kKeysPerStep; ++u) {
                 if (tok + u < end) {
                     float k[DPL];
-                    load_bf16<DPL>(kbase + (int64_t)(tok + u) * D, k);
-                    load_bf16<DPL>(vbase + (int64_t)(tok + u) * D, v[u]);
+                    load_bf16<DPL>(kb + (int64_t)(tok + u) * tstride, k);
+                    load_bf16<DPL>(vb + (int64_t)(tok + u) * tstride, v[u]);
                     float acc = 0.f;
 #pragma unroll
                     for (int d = 0; d < DPL; ++d) acc = fmaf(q[d], k[d], acc);
@@ -142,8 +148,13 @@ attend_simt_kernel(const __nv_bfloat16* __restrict__ Q, int64_t q_row, int64_t q
 
 cudaError_t launch_attend_simt(const Strided& Q, const Strided& O, const LayerRegion& region, const RangeList& ranges,
                                int32_t T, int32_t rows, int32_t heads, int32_t D, float softmax_scale,
-                               cudaStream_t stream)
+                               cudaStream_t stream, const CurrentScaleSource* cur)
 {
+    const __nv_bfloat16* ek = cur ? (const __nv_bfloat16*)cur->K.ptr : nullptr;
+    const __nv_bfloat16* ev = cur ? (const __nv_bfloat16*)cur->V.ptr : nullptr;
+    const int64_t e_row = cur ? cur->K.row : 0, e_head = cur ? cur->K.head : 0, e_tok = cur ? cur->K.token : 0;
+    const int ext_range = cur ? ranges.n - 1 : -1;
+    if (cur && (cur->store || cur->V.row != e_row || cur->V.head != e_head || cur->V.token != e_tok)) return cudaErrorNotSupported;
     const int64_t total_rows = (int64_t)rows * heads * T;
     if (total_rows == 0) return cudaSuccess;
     const int64_t threads = total_rows * kLanesPerRow;
@@ -153,11 +164,11 @@ cudaError_t launch_attend_simt(const Strided& Q, const Strided& O, const LayerRe
     if (D == 64) {
         attend_simt_kernel<64><<<(unsigned)blocks, kThreads, 0, stream>>>(
             (const __nv_bfloat16*)Q.ptr, Q.row, Q.head, Q.token, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token,
-            region.base, region.capacity, ranges, T, heads, total_rows, scale_log2);
+            region.base, region.capacity, ranges, T, heads, total_rows, scale_log2, ek, ev, e_row, e_head, e_tok, ext_range);
     } else {
         attend_simt_kernel<128><<<(unsigned)blocks, kThreads, 0, stream>>>(
             (const __nv_bfloat16*)Q.ptr, Q.row, Q.head, Q.token, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token,
-            region.base, region.capacity, ranges, T, heads, total_rows, scale_log2);
+            region.base, region.capacity, ranges, T, heads, total_rows, scale_log2, ek, ev, e_row, e_head, e_tok, ext_range);
     }
     count_launch();
     return cudaGetLastError();

@@ -565,13 +565,9 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
                    int3 qpos, float scale_log2, int* status, int sm_count, cudaStream_t stream)
 {
     using C = Cfg<D>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static SharedMemoryOptIn opt_in;
+    const cudaError_t oe = opt_in.ensure(attend_tc_kernel<D>, (int)C::kSmemBytes);
+    if (oe != cudaSuccess) return oe;
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > units) grid = units;
     attend_tc_kernel<D><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(

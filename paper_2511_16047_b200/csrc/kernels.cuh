@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 
 #include "policy.hpp"
@@ -45,9 +46,20 @@ cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion&
                           int32_t T, int32_t rows, int32_t heads, int32_t D, bool bulk, int* status, int sm_count,
                           cudaStream_t stream);
 
+// The current scale taken from the caller's K/V tensors instead of the cache: the last entry of the
+// range list given with it stands for that scale (start 0, len T).  With `store`, the kernel also
+// writes the scale to position `dst` of every item's part of `region` (the append fused into attention).
+struct CurrentScaleSource {
+    Strided K, V;
+    bool store;
+    int32_t dst;
+    LayerRegion region;
+};
+
+// (the CUDA-core kernel takes a current-scale source without `store` only)
 cudaError_t launch_attend_simt(const Strided& Q, const Strided& O, const LayerRegion& region, const RangeList& ranges,
                                int32_t T, int32_t rows, int32_t heads, int32_t D, float softmax_scale,
-                               cudaStream_t stream);
+                               cudaStream_t stream, const CurrentScaleSource* cur = nullptr);
 
 constexpr int kSimilarityMaxBlocks = 2048;
 cudaError_t launch_similarity(const __nv_bfloat16* K_prev, int32_t side_prev, const __nv_bfloat16* K_cur,
@@ -73,16 +85,6 @@ bool tc_encode_q_map(const Strided& Q, int32_t T, int32_t rows, int32_t heads, i
 bool tc_encode_kv_store_maps(const LayerRegion& region, int64_t items, int32_t D, int box_rows, int32_t token_extent,
                              void* k_map_out, void* v_map_out);
 
-// The current scale taken from the caller's K/V tensors instead of the cache: the last entry of the
-// range list given with it stands for that scale (start 0, len T).  With `store`, the kernel also
-// writes the scale to position `dst` of every item's part of `region` (the append fused into attention).
-struct CurrentScaleSource {
-    Strided K, V;
-    bool store;
-    int32_t dst;
-    LayerRegion region;
-};
-
 // Paired tensor-core kernel: two softmax groups per CTA, probabilities kept in tensor memory.
 cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map16, const void* v_map16,
                                const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
@@ -98,5 +100,22 @@ cudaError_t launch_attend_small(const Strided& Q, const Strided& O, const LayerR
                                 cudaStream_t stream);
 
 void count_launch(int n = 1);
+
+// A kernel's dynamic shared-memory limit is a per-device setting: raised once per device and kernel,
+// from whichever host thread gets there first (setting it twice is harmless).
+struct SharedMemoryOptIn {
+    std::atomic<uint64_t> done{0};   // bit d: set on device d
+    template <typename Kernel>
+    cudaError_t ensure(Kernel* kernel, int bytes)
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1u)) return cudaSuccess;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess && dev >= 0 && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+        return e;
+    }
+};
 
 }  // namespace amskv

@@ -34,9 +34,12 @@ struct TokenRun {
 // right-aligned and slot 1 directly above the pinned region, which makes the resident
 // tokens one contiguous run whenever w <= 2.
 struct LayerLayout {
+    static constexpr int32_t kMinCapacity = 16;   // with a never-stored last scale a region could be empty; its tensor maps need an extent
     int32_t c = 0;          // pinned scales (clamped to the schedule length)
     int32_t w = 1;          // window, in scales (clamped)
     bool full = false;      // nothing is ever evicted
+    bool skip_last = false; // the last scale of the schedule is never stored (no later scale reads it)
+    int32_t n_scales = 0;
     int32_t capacity = 0;   // tokens per item
     std::vector<int32_t> offset;  // [n_scales] token offset of each segment's home
 
@@ -55,31 +58,35 @@ struct LayerLayout {
     std::vector<uint8_t> transient;   // [n_scales] scale is read from the transient slot at its own step
     std::vector<int64_t> stream_end;  // [n_scales] stream length after the scale
 
-    void build(const std::vector<int32_t>& tokens, int32_t n_condensed, int32_t n_local, bool demanding)
+    void build(const std::vector<int32_t>& tokens, int32_t n_condensed, int32_t n_local, bool demanding,
+               bool transient_last = false)
     {
         const int32_t K = (int32_t)tokens.size();
+        n_scales = K;
+        skip_last = transient_last;
+        const int32_t stored = skip_last ? K - 1 : K;   // scales that get a home
         c = std::min(std::max(n_condensed, 0), K);
         w = std::min(std::max(n_local, 1), K);
         full = demanding || (c + w >= K);
         offset.assign(K, 0);
         if (full) {
             int32_t at = 0;
-            for (int32_t s = 0; s < K; ++s) { offset[s] = at; at += tokens[s]; }
-            capacity = at;
+            for (int32_t s = 0; s < stored; ++s) { offset[s] = at; at += tokens[s]; }
+            capacity = skip_last ? std::max(at, kMinCapacity) : at;
             return;
         }
         std::vector<int32_t> slot_size(w, 0);
-        for (int32_t s = c; s < K; ++s) slot_size[(s - c) % w] = std::max(slot_size[(s - c) % w], tokens[s]);
+        for (int32_t s = c; s < stored; ++s) slot_size[(s - c) % w] = std::max(slot_size[(s - c) % w], tokens[s]);
         int32_t pinned = 0;
         for (int32_t s = 0; s < c; ++s) pinned += tokens[s];
         const int32_t pinned_at = slot_size[0];
         std::vector<int32_t> slot_at(w, 0);
         int32_t at = pinned_at + pinned;
         for (int32_t j = 1; j < w; ++j) { slot_at[j] = at; at += slot_size[j]; }
-        capacity = at;
+        capacity = skip_last ? std::max(at, kMinCapacity) : at;
         int32_t p = pinned_at;
         for (int32_t s = 0; s < c; ++s) { offset[s] = p; p += tokens[s]; }
-        for (int32_t s = c; s < K; ++s) {
+        for (int32_t s = c; s < stored; ++s) {
             const int32_t j = (s - c) % w;
             offset[s] = (j == 0) ? (slot_size[0] - tokens[s]) : slot_at[j];
         }
@@ -88,9 +95,11 @@ struct LayerLayout {
     // Token-budget form: `budget` = C_bgt (C_max for a cache-demanding layer, C_min otherwise) and
     // `condensed` = C_cds, both in tokens.  Starting a cache-demanding layer at C_max is the same as
     // promoting it at its first overflow, because nothing is evicted before that overflow.
-    void build_tokens(const std::vector<int32_t>& tokens, int32_t budget, int32_t condensed)
+    void build_tokens(const std::vector<int32_t>& tokens, int32_t budget, int32_t condensed, bool transient_last = false)
     {
         const int32_t K = (int32_t)tokens.size();
+        n_scales = K;
+        skip_last = transient_last;
         token_mode = true;
         full = false;
         c = 0;
@@ -115,11 +124,13 @@ struct LayerLayout {
             } else {
                 transient[s] = 1;  // never cached (Algorithm 1 skips it); attended from the transient slot
             }
-            if (transient[s]) slot = std::max(slot, T);
+            if (transient[s] && !(skip_last && s == K - 1)) slot = std::max(slot, T);
             stream_end[s] = g;
         }
-        used = (int32_t)std::min<int64_t>(g, c_bgt);
-        capacity = used + slot;
+        // (a last scale that is never stored takes no room: neither in the ring nor in the transient slot)
+        const int64_t stored_stream = skip_last ? (K > 1 ? stream_end[K - 2] : 0) : g;
+        used = (int32_t)std::min<int64_t>(stored_stream, c_bgt);
+        capacity = skip_last ? std::max(used + slot, kMinCapacity) : used + slot;
     }
 
     int32_t position(int64_t g) const
@@ -138,6 +149,7 @@ struct LayerLayout {
     bool keeps(int32_t s, int32_t k) const
     {
         if (s > k) return false;
+        if (skip_last && s == n_scales - 1) return false;   // attended at its own step, never held
         if (!token_mode) return full || s < c || s > k - w;
         if (!cached[s]) return false;
         const int64_t e = stream_end[s], b = s > 0 ? stream_end[s - 1] : 0;
@@ -170,6 +182,7 @@ struct LayerLayout {
     int32_t pieces(const std::vector<int32_t>& tokens, int32_t k, Piece* out) const
     {
         const int32_t T = tokens[k];
+        if (skip_last && k == n_scales - 1) return 0;
         if (!token_mode) {
             out[0] = Piece{0, offset[k], T};
             return 1;
@@ -198,6 +211,7 @@ struct LayerLayout {
     // token ranges read at scale k, sorted by position and merged where they touch
     int32_t ranges(const std::vector<int32_t>& tokens, int32_t k, Range* out) const
     {
+        if (skip_last && k == n_scales - 1) return ranges_before(tokens, k, out);   // the scale itself is not in the cache
         if (token_mode) {
             int32_t n = 0;
             int32_t res = (int32_t)std::min<int64_t>(stream_end[k], c_bgt);
@@ -229,13 +243,13 @@ struct LayerLayout {
         int32_t n = 0;
         if (!token_mode) {
             for (int32_t s = 0; s <= k; ++s)
-                if (keeps(s, k)) out[n++] = TokenRun{s, 0, tokens[s]};
+                if (s == k || keeps(s, k)) out[n++] = TokenRun{s, 0, tokens[s]};
             return n;
         }
         const bool rolled = stream_end[k] > c_bgt;
         const int64_t lo = tail_begin(k);
         for (int32_t s = 0; s <= k; ++s) {
-            if (!cached[s] || (s == k && transient[k])) continue;
+            if (!cached[s] || (s == k && (transient[k] || (skip_last && k == n_scales - 1)))) continue;
             const int64_t e = stream_end[s], b = e - tokens[s];
             if (!rolled) {
                 out[n++] = TokenRun{s, 0, tokens[s]};
@@ -249,7 +263,7 @@ struct LayerLayout {
                 else out[n++] = TokenRun{s, (int32_t)(t0 - b), (int32_t)(e - t0)};
             }
         }
-        if (transient[k]) out[n++] = TokenRun{k, 0, tokens[k]};
+        if (transient[k] || (skip_last && k == n_scales - 1)) out[n++] = TokenRun{k, 0, tokens[k]};
         return n;
     }
 
@@ -289,6 +303,15 @@ struct LayerLayout {
 
     int64_t resident_tokens(const std::vector<int32_t>& tokens, int32_t k) const
     {
+        if (skip_last && k == n_scales - 1) {
+            // what the step leaves in the cache: the older tokens its queries attended to
+            TokenRun runs[2 * 32];
+            const int32_t n_runs = attended(tokens, k, runs);
+            int64_t t = 0;
+            for (int32_t i = 0; i < n_runs; ++i)
+                if (runs[i].segment != k) t += runs[i].count;
+            return t;
+        }
         if (token_mode) return std::min<int64_t>(stream_end[k], c_bgt);
         int64_t t = 0;
         for (int32_t s = 0; s <= k; ++s)
