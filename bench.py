@@ -313,17 +313,33 @@ def run_ours(args):
     e2e = None
     if not args.no_e2e:
         nst = B.amskv_step_staging_bytes(cache)
-        staging = torch.empty(nst, dtype=torch.uint8, device="cuda")
+        # Two staging buffers on two streams, calls alternating between them: the device-to-host copy of one
+        # call's result overlaps the host-to-device copies of the next call (the link is full duplex), and a
+        # kernel can run while the other stream copies.  Per layer the calls stay ordered by events.
+        stagings = [torch.empty(nst, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        lanes = [torch.cuda.Stream(), torch.cuda.Stream()]
+        layer_done = [torch.cuda.Event() for _ in range(wl.layers)]
         hq = [q.cpu().pin_memory() for q, _, _ in qkv]
         hk = [k.cpu().pin_memory() for _, k, _ in qkv]
         hv = [v.cpu().pin_memory() for _, _, v in qkv]
-        ho = [torch.empty_like(q).pin_memory() for q in hq]
+        # one result buffer per lane and scale: a call's result is read back while the next call runs
+        ho = [[torch.empty_like(q).pin_memory() for q in hq] for _ in range(2)]
 
         def host_step():
             B.amskv_cache_reset(cache)
+            for lane in lanes:
+                lane.wait_stream(stream)
+            i = 0
             for k in range(K):
                 for layer in range(wl.layers):
-                    B.amskv_step_host(cache, layer, k, hk[k], hv[k], hq[k], ho[k], staging, nst, stream)
+                    lane = i & 1
+                    if k > 0:
+                        lanes[lane].wait_event(layer_done[layer])   # the layer's previous scale (maybe on the other lane)
+                    B.amskv_step_host(cache, layer, k, hk[k], hv[k], hq[k], ho[lane][k], stagings[lane], nst, lanes[lane])
+                    layer_done[layer].record(lanes[lane])
+                    i += 1
+            for lane in lanes:
+                stream.wait_stream(lane)
 
         host_step()
         torch.cuda.synchronize()
@@ -345,7 +361,7 @@ def run_ours(args):
         d2h = wl.layers * sum(q.numel() * 2 for q in hq)
         e2e = {"value": e_ms * 1e3 / (wl.batch * world) , "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e_steps, "ms_per_step": e_ms}
-        del staging, hq, hk, hv, ho
+        del stagings, hq, hk, hv, ho
     B.amskv_cache_destroy(cache)
     del arena
     torch.cuda.empty_cache()
