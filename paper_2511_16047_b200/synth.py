@@ -18,6 +18,9 @@ import torch
 # (Sec. 3.2); the 1024x1024 text-to-image schedule ends at 64x64.
 SIDES_256 = (1, 2, 3, 4, 5, 6, 8, 10, 13, 16)
 SIDES_1024 = (1, 2, 4, 6, 8, 12, 16, 20, 24, 32, 40, 48, 64)
+# 512x512 class-conditional generation (Sec. 5 evaluates a depth-36 model on it): the paper does not
+# print that schedule; this is a ten-scale schedule ending at 32x32 (2 240 tokens) of the same kind.
+SIDES_512 = (1, 2, 3, 4, 6, 9, 13, 18, 24, 32)
 
 
 @dataclasses.dataclass(frozen=True)
@@ -78,6 +81,8 @@ WORKLOADS = {
     "var_d16": Workload("var_d16", 16, 16, 64, 64, SIDES_256, 2, 2, 0.5, 20251117),
     # VAR-d30-shaped: dim 1920, batch 256 (the batch the paper reaches only with AMS-KV)
     "var_d30": Workload("var_d30", 30, 30, 64, 256, SIDES_256, 2, 2, 0.3, 20251118),
+    # depth-36-shaped 512x512 model: dim 2304 = 36 heads x 64, 36 layers, batch 32
+    "var_d36_512": Workload("var_d36_512", 36, 36, 64, 32, SIDES_512, 2, 2, 0.3, 20251120),
     # 1024x1024 text-to-image shaped: dim 2048, head_dim 128, batch 8
     "t2i_1024": Workload("t2i_1024", 32, 16, 128, 8, SIDES_1024, 3, 2, 0.4, 20251119),
 }

@@ -71,6 +71,13 @@ def test_text_to_image_1024_shape_sampled():
     _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 3, seed=12, need_gb=3.0)
 
 
+def test_depth_36_512_shape_sampled():
+    """36 heads x 64 (dim 2304), ten scales up to 32 x 32 (2 240 tokens): head_dim 64 with eight query
+    tiles per item at the last scale, one layer of each class, sampled items and query rows."""
+    wl = synth.WORKLOADS["var_d36_512"].replace(batch=8)
+    _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 6, seed=14, need_gb=3.0)
+
+
 @pytest.mark.parametrize("batch", [1, 16])
 def test_policy_sweep_on_var_d30_shape(batch):
     """The VAR-d30 head layout at small batches with a mix of condensed / local settings and layer
