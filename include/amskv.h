@@ -196,8 +196,8 @@ AMSKV_API int amskv_attend(amskv_cache* cache, int layer, int scale, const void*
  * the scale's place in the cache on the way -- the separate copy and its second read of K and V
  * disappear.  Scales served by the other attention kernels, appends that are more than one
  * contiguous copy (a token budget whose ring wraps inside the scale) and, under AMSKV_PATH_AUTO,
- * scales where splitting the current scale off its cache range would add a 64-token key tile, run
- * as the two calls.
+ * scales of fewer than 64 tokens and scales where splitting the current scale off its cache range
+ * would add a 64-token key tile, run as the two calls.
  *   K, V: as for amskv_append (one stride triple kv_strides for both); Q, out: as for
  *   amskv_attend.  out must not alias K or V.
  * Stream ordering: as for the two calls -- this call must come after attend(layer, scale - 1)
