@@ -207,6 +207,25 @@ AMSKV_API int amskv_append_attend(amskv_cache* cache, int layer, int scale, cons
                                   const int64_t kv_strides[3], const void* Q, void* out, const int64_t q_strides[3],
                                   const int64_t o_strides[3], void* stream);
 
+/*
+ * Attention density (Sec. 4.1): d = (1 / T_i) * sum over the queries of `scale` and over the keys of a
+ * retained scale i of the attention probabilities -- the attention a retained scale receives per key
+ * token, the quantity behind the choice of the condensed and local scales.  An analysis call, not part
+ * of the generation step; it recomputes the softmax of amskv_attend(layer, scale, Q) on the CUDA cores
+ * (fp32, no rounding of the probabilities).
+ *   out          device pointer to heads * n doubles, n = the number of runs amskv_attended_tokens
+ *                reports for (layer, scale); out[h * n + r] receives the density of run r for head h,
+ *                averaged over the rows.  For a run that is part of a segment (token budgets) the
+ *                divisor is the run's own token count.  Zeroed and filled by the call, on `stream`.
+ *   out_entries  doubles `out` can hold (NOMEM if too few).
+ * `scale` must be the scale most recently appended to `layer` (ORDER otherwise); a never-stored last
+ * scale is refused (UNSUPPORTED: its keys are not in the cache).  The sums are accumulated with
+ * floating-point atomic adds, so results agree to rounding only between calls.
+ * Identity: sum over r of count_r * out[h * n + r] = T of `scale` (every query's probabilities sum to 1).
+ */
+AMSKV_API int amskv_attention_density(amskv_cache* cache, int layer, int scale, const void* Q,
+                                      const int64_t q_strides[3], double* out, size_t out_entries, void* stream);
+
 /* Choose the kernel used by amskv_attend (AMSKV_PATH_*).  The default is AUTO. */
 AMSKV_API int amskv_set_attend_path(amskv_cache* cache, int path);
 

@@ -114,6 +114,31 @@ def attend_tokens(Q, K_segments: Sequence, V_segments: Sequence, tokens: Sequenc
     return attention(Q, np.concatenate(k_parts, axis=1), np.concatenate(v_parts, axis=1), scale)
 
 
+def attention_density(Q, K_segments: Sequence, runs: Sequence, scale: float, heads: int) -> np.ndarray:
+    """Attention density (Sec. 4.1) of the queries Q over runs of retained keys.
+
+    Q: [n, T, D] with n = rows * heads (item = row * heads + head); K_segments[s]: [n, T_s, D];
+    runs: (segment, first token, count) triples.  P = softmax(scale * Q Kc^T) over the concatenated
+    keys of all runs; the density of a run is the sum of P over all queries and over the run's keys,
+    divided by the run's token count; the result [heads, len(runs)] is the mean over rows.
+    """
+    Q = _f64(Q)
+    n, T, D = Q.shape
+    Kc = np.concatenate([_f64(K_segments[s])[:, first:first + count, :] for s, first, count in runs], axis=1)
+    logits = scale * np.einsum("ntd,nld->ntl", Q, Kc)
+    logits -= logits.max(axis=2, keepdims=True)
+    P = np.exp(logits)
+    P /= P.sum(axis=2, keepdims=True)
+    out = np.zeros((heads, len(runs)), dtype=np.float64)
+    rows = n // heads
+    at = 0
+    for r, (_, _, count) in enumerate(runs):
+        mass = P[:, :, at:at + count].sum(axis=(1, 2)) / count      # per item
+        out[:, r] = mass.reshape(rows, heads).mean(axis=0)
+        at += count
+    return out
+
+
 def block_causal_attention(Q_all, K_all, V_all, sides: Sequence[int], scale: float) -> np.ndarray:
     """Vanilla next-scale attention over all tokens at once with the scale-block mask."""
     Q_all, K_all, V_all = _f64(Q_all), _f64(K_all), _f64(V_all)

@@ -62,6 +62,7 @@ def _load() -> ctypes.CDLL:
         "amskv_append": ([vp, i, i, vp, vp, i64p, vp], i),
         "amskv_attend": ([vp, i, i, vp, vp, i64p, i64p, vp], i),
         "amskv_append_attend": ([vp, i, i, vp, vp, i64p, vp, vp, i64p, i64p, vp], i),
+        "amskv_attention_density": ([vp, i, i, vp, i64p, vp, sz, vp], i),
         "amskv_set_attend_path": ([vp, i], i),
         "amskv_step_host": ([vp, i, i, vp, vp, vp, vp, vp, sz, vp], i),
         "amskv_step_staging_bytes": ([vp, szp], i),
@@ -89,7 +90,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy amskv_cache_reset amskv_append "
-           "amskv_attend amskv_append_attend amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
+           "amskv_attend amskv_append_attend amskv_attention_density amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
            "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
            "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_attended_tokens amskv_append_copies "
            "amskv_cache_bytes amskv_status "
@@ -190,6 +191,12 @@ def amskv_append_attend(cache: int, layer: int, scale: int, K, V, Q, out, stream
         raise ValueError("K and V must share one stride triple")
     _check(lib.amskv_append_attend(cache, layer, scale, _addr(K), _addr(V), ks, _addr(Q), _addr(out), _strides(Q),
                                    _strides(out), _stream(stream)), "amskv_append_attend")
+
+
+def amskv_attention_density(cache: int, layer: int, scale: int, Q, out, out_entries: int, stream=None) -> None:
+    """Attention density per (head, run of amskv_attended_tokens) into `out` (device doubles)."""
+    _check(lib.amskv_attention_density(cache, layer, scale, _addr(Q), _strides(Q), _addr(out), int(out_entries),
+                                       _stream(stream)), "amskv_attention_density")
 
 
 def amskv_set_attend_path(cache: int, path: int) -> None:

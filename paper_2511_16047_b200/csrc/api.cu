@@ -428,6 +428,38 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
     return AMSKV_OK;
 }
 
+int amskv_attention_density(amskv_cache* cache, int layer, int scale, const void* Q, const int64_t q_strides[3],
+                            double* out, size_t out_entries, void* stream)
+{
+    if (bad_layer_scale(cache, layer, scale) || !out || (reinterpret_cast<uintptr_t>(out) & 7u)) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
+    if (scale != cache->last_appended[layer]) return AMSKV_ERR_ORDER;
+    const int32_t T = cache->tokens[scale];
+    Strided q;
+    int rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
+    if (rc != AMSKV_OK) return rc;
+    const LayerLayout& lay = cache->layout[layer];
+    TokenRun runs[2 * AMSKV_MAX_SCALES];
+    const int32_t n_runs = lay.attended(cache->tokens, scale, runs);
+    if (out_entries < (size_t)cache->heads * (size_t)n_runs) return AMSKV_ERR_NOMEM;
+    LayerLayout::RunPiece rp[kMaxDensityPieces];
+    const int32_t n = lay.attended_pieces(cache->tokens, scale, rp, kMaxDensityPieces);
+    if (n < 0) return AMSKV_ERR_UNSUPPORTED;   // the scale's own keys are not in the cache (never-stored last scale)
+    DensityPieces pieces;
+    pieces.n = n;
+    pieces.n_runs = n_runs;
+    for (int32_t i = 0; i < n; ++i) {
+        pieces.start[i] = rp[i].start;
+        pieces.len[i] = rp[i].len;
+        pieces.run[i] = rp[i].run;
+        pieces.weight[i] = 1.0 / (double)runs[rp[i].run].count;
+    }
+    cudaError_t e = launch_density(q, cache->region(layer), pieces, T, cache->rows, cache->heads, cache->head_dim,
+                                   cache->softmax_scale, out, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
+}
+
 int amskv_step_staging_bytes(const amskv_cache* cache, size_t* bytes)
 {
     if (!cache || !bytes) return AMSKV_ERR_INVALID;

@@ -99,6 +99,17 @@ cudaError_t launch_attend_small(const Strided& Q, const Strided& O, const LayerR
                                 int32_t T, int32_t rows, int32_t heads, int32_t D, float softmax_scale,
                                 cudaStream_t stream);
 
+// Attention density: the pieces of the per-item region that hold the attended tokens, each with the run
+// (of the attended-token list) it belongs to and the weight 1 / (tokens of that run).
+constexpr int kMaxDensityPieces = 96;
+struct DensityPieces {
+    int32_t n, n_runs;
+    int32_t start[kMaxDensityPieces], len[kMaxDensityPieces], run[kMaxDensityPieces];
+    double weight[kMaxDensityPieces];
+};
+cudaError_t launch_density(const Strided& Q, const LayerRegion& region, const DensityPieces& pieces, int32_t T,
+                           int32_t rows, int32_t heads, int32_t D, float softmax_scale, double* out, cudaStream_t stream);
+
 void count_launch(int n = 1);
 
 // A kernel's dynamic shared-memory limit is a per-device setting: raised once per device and kernel,

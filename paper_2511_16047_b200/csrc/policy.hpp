@@ -301,6 +301,40 @@ struct LayerLayout {
         return n;
     }
 
+    // Where the runs of attended(k) sit in the per-item region right after the append of scale k: pieces
+    // (start, len) tagged with the index of their run; a run of a token-budget layer is two pieces where
+    // the ring wraps inside it.  Returns the number of pieces, or -1 if a run has no place in the region
+    // (a never-stored last scale) or `cap` is too small.
+    struct RunPiece {
+        int32_t start, len, run;
+    };
+    int32_t attended_pieces(const std::vector<int32_t>& tokens, int32_t k, RunPiece* out, int32_t cap) const
+    {
+        TokenRun runs[2 * 32];
+        const int32_t n_runs = attended(tokens, k, runs);
+        int32_t n = 0;
+        for (int32_t i = 0; i < n_runs; ++i) {
+            const int32_t s = runs[i].segment;
+            if (skip_last && s == n_scales - 1) return -1;
+            if (!token_mode || (s == k && transient[k])) {
+                if (n >= cap) return -1;
+                out[n++] = RunPiece{(token_mode ? used : offset[s]) + runs[i].first, runs[i].count, i};
+                continue;
+            }
+            int64_t g = (s > 0 ? stream_end[s - 1] : 0) + runs[i].first;
+            int32_t left = runs[i].count;
+            while (left > 0) {
+                const int32_t p = g < c_cds ? (int32_t)g : position(g);
+                const int32_t run = std::min<int32_t>(left, (g < c_cds ? c_cds : c_bgt) - p);
+                if (n >= cap) return -1;
+                out[n++] = RunPiece{p, run, i};
+                g += run;
+                left -= run;
+            }
+        }
+        return n;
+    }
+
     int64_t resident_tokens(const std::vector<int32_t>& tokens, int32_t k) const
     {
         if (skip_last && k == n_scales - 1) {
