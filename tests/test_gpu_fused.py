@@ -37,7 +37,8 @@ def test_single_layer_every_element_every_scale(path, fused):
         assert B.amskv_cache_bytes(c.h)[1] == oracle.kv_bytes(wl.sides, pols, wl.rows, wl.heads, wl.head_dim)
 
 
-def test_cache_contents_equal_those_of_the_separate_calls():
+@pytest.mark.parametrize("path", [B.PATH_TENSOR_PAIR, B.PATH_AUTO, B.PATH_SMALL], ids=["pair", "auto", "small"])
+def test_cache_contents_equal_those_of_the_separate_calls(path):
     """Byte-for-byte: the arena after a fused pass equals the arena after append + attend."""
     _need()
     sides, rows, heads, D = (1, 2, 3, 5, 7, 9, 12, 17), 3, 5, 64
@@ -47,7 +48,7 @@ def test_cache_contents_equal_those_of_the_separate_calls():
     for fused in (False, True):
         with Cache(len(pols), heads, D, rows, sides, pols) as c:
             c.arena.zero_()
-            run_pass(c, qkv, B.PATH_TENSOR_PAIR, fused=fused)
+            run_pass(c, qkv, path, fused=fused)
             arenas.append(c.arena[256:].clone())
     assert torch.equal(arenas[0], arenas[1])
 
