@@ -73,13 +73,17 @@ struct Barriers {
 
 static_assert(sizeof(Barriers) + 1024 <= 4096, "barrier block must fit in front of the 1024-byte aligned tiles");
 
-// How the pairs of one launch are formed; shared by every role.
+// How the pairs (units of two streams) of one launch are formed; shared by every role.  The first
+// n_shared pairs are two consecutive query tiles of one item, which share every key/value tile in
+// shared memory; an item with an odd number of query tiles has one tile left over, and the left-over
+// tiles of two consecutive items form a pair whose streams fetch their own key/value tiles (with one
+// query tile per item every pair is of that kind).
 struct PairPlan {
-    int32_t two_q;        // 1: streams are query tiles of one item; 0: streams are two items
     int32_t nqt;          // query tiles per item
-    int32_t npi;          // pairs per item (two_q) -- else unused
+    int32_t npi;          // shared pairs per item = nqt / 2
     int32_t n_items;
-    int32_t n_pairs;
+    int32_t n_shared;     // = n_items * npi
+    int32_t n_pairs;      // n_shared + ceil(n_items * (nqt & 1) / 2)
 };
 
 // The current scale read from the caller's K/V tensors instead of the cache: the last entry of the
@@ -101,16 +105,18 @@ struct Stream {
     bool valid;
 };
 
+__device__ __forceinline__ bool pair_is_shared(const PairPlan& pp, int32_t pair) { return pair < pp.n_shared; }
+
 __device__ __forceinline__ Stream stream_of(const PairPlan& pp, int32_t pair, int g)
 {
     Stream s;
-    if (pp.two_q) {
+    if (pair < pp.n_shared) {
         s.item = pp.npi == 1 ? pair : pair / pp.npi;
         s.qt = 2 * (pair - s.item * pp.npi) + g;
-        s.valid = s.qt < pp.nqt;
+        s.valid = true;
     } else {
-        s.item = 2 * pair + g;
-        s.qt = 0;
+        s.item = 2 * (pair - pp.n_shared) + g;
+        s.qt = pp.nqt - 1;
         s.valid = s.item < pp.n_items;
     }
     return s;
@@ -535,9 +541,10 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (uint32_t n = 0; ok && n < my_pairs; ++n) {
             const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
             const Stream sa = stream_of(pp, pair, 0), sb = stream_of(pp, pair, 1);
-            const int per_tile = (!pp.two_q && sb.valid) ? 2 : 1;
-            // one unit per item writes the item's tiles: with two query tiles per unit, the unit of the first tiles
-            const bool unit_stores = storing && (!pp.two_q || sa.qt == 0);
+            const bool shared = pair_is_shared(pp, pair);
+            const int per_tile = (!shared && sb.valid) ? 2 : 1;
+            // one unit per item writes the item's tiles: the unit of its first query tiles
+            const bool unit_stores = storing && (shared ? sa.qt == 0 : pp.nqt == 1);
             for (int j = 0; ok && j < n_tiles; ++j) {
                 int32_t t0, valid;
                 tile_of(j, t0, valid);
@@ -681,6 +688,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             for (uint32_t n = 0; ok && n < my_pairs; ++n) {
                 const int32_t pair = (int32_t)(blockIdx.x + n * gridDim.x);
                 const int ng = stream_of(pp, pair, 1).valid ? 2 : 1;
+                const bool shared = pair_is_shared(pp, pair);
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     int32_t t0, valid;
                     tile_of(j, t0, valid);
@@ -700,7 +708,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         }
                         // S = Q K^T for (stream g, tile j).  Its operands are waited for first: they have
                         // almost always landed, and this keeps the two waits out of the P -> P V -> S chain.
-                        const uint32_t seq = pp.two_q ? sq : sq + g;
+                        const uint32_t seq = shared ? sq : sq + g;
                         const uint32_t stage = seq % C::kStages, use = seq / C::kStages;
                         if (j == 0) {
                             const uint32_t u = ucount[g];
@@ -709,7 +717,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                             if (!warp_wait(q_full0 + 16 * g + 8 * q_half[g], parity, abort_flag)) { ok = false; continue; }
                             ++ucount[g];
                         }
-                        if (!(pp.two_q && g == 1)) {  // the second stream of a shared tile finds it landed already
+                        if (!(shared && g == 1)) {  // the second stream of a shared tile finds it landed already
                             if (!warp_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) { ok = false; continue; }
                         }
                         if (pv_live[g] && !issue_pv(g)) { ok = false; continue; }
@@ -733,10 +741,10 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         pv_nch[g] = nch;
                         pv_first[g] = (j == 0);
                         pv_last[g] = (j == n_tiles - 1);
-                        pv_release[g] = pp.two_q ? (g == ng - 1) : true;
+                        pv_release[g] = shared ? (g == ng - 1) : true;
                         ++tcount[g];
                     }
-                    sq += pp.two_q ? 1 : ng;
+                    sq += shared ? 1 : ng;
                 }
             }
 #pragma unroll
@@ -1000,11 +1008,14 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     memcpy(&vm64, v_map64, sizeof(vm64));
     PairPlan pp;
     pp.nqt = (T + kQRows - 1) / kQRows;
-    pp.two_q = pp.nqt >= 2 ? 1 : 0;
-    pp.npi = (pp.nqt + 1) / 2;
+    pp.npi = pp.nqt / 2;
     if ((int64_t)rows * heads > 0x3fffffffll) return cudaErrorInvalidValue;
     pp.n_items = rows * heads;
-    pp.n_pairs = pp.two_q ? pp.n_items * pp.npi : (pp.n_items + 1) / 2;
+    const int64_t n_shared = (int64_t)pp.n_items * pp.npi;
+    const int64_t n_pairs = n_shared + ((pp.nqt & 1) ? ((int64_t)pp.n_items + 1) / 2 : 0);
+    if (n_pairs > 0x7fffffffll) return cudaErrorInvalidValue;
+    pp.n_shared = (int32_t)n_shared;
+    pp.n_pairs = (int32_t)n_pairs;
     int32_t n_tiles = 0;
     for (int i = 0; i < ranges.n; ++i) n_tiles += (ranges.r[i].len + kKT - 1) / kKT;
     const int3 qpos = make_int3(pos[0], pos[1], pos[2]);
