@@ -36,16 +36,19 @@ constexpr int kKT = 64;           // key/value tokens per tile
 constexpr int kKVBoxRows = 16;    // tokens per bulk copy
 constexpr int kGroupWarps = 4;
 constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp = 9;
-constexpr int kThreads = 320;
+constexpr int kMmaWarp = 9;        // first MMA-issuing warp; Cfg<D>::kMmaWarps of them
 constexpr int kMaxStages = 4;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleLog2 = 8.f;
 constexpr int kQSplitRows = 64;   // query tiles of at most this many rows are double-buffered inside their slot
 constexpr int kPolyEvery = 4;     // every 4th pair of exponentials goes to the FMA pipe (0: none)
 
-template <int D>
+// kWide: one CTA per SM with two S buffers per stream and an issuing warp per stream (below): the form
+// 128 channels use.  64 channels use the two-CTA form (the wide form is instantiable for them, but lost
+// wherever it was measured).
+template <int D, bool kWide>
 struct Cfg {
+    static_assert(D == 64 || kWide, "128 channels always use the wide form");
     static constexpr int kHalves = D / 64;                      // 128-byte swizzle atoms per row
     static constexpr int kStages = 4;
     static constexpr uint32_t kQBytes = kQRows * D * 2;         // one query tile
@@ -55,9 +58,20 @@ struct Cfg {
     static constexpr uint32_t kStageBytes = 2 * kKVBytes;
     static constexpr uint32_t kTileBytes = 2 * kQBytes + kStages * kStageBytes;
     static constexpr uint32_t kSmemBytes = 4096 + kTileBytes;   // barriers, tile table and alignment slack in front
-    static constexpr uint32_t kTmemCols = (D == 64) ? 256 : 512;  // S x2 (64 each) + O x2 (D each)
-    static constexpr uint32_t kSCol = 0, kOCol = 2 * kKT;
-    static constexpr int kCtasPerSm = (D == 64) ? 2 : 1;
+    // Score buffers per stream.  With 64 channels two CTAs share the SM's 512 tensor-memory columns and a
+    // stream has one S buffer (S and O of two streams: 256 columns).  With 128 channels one CTA has all
+    // 512 columns and a stream has two S buffers used alternately, so that S of the next tile is computed
+    // while the softmax of the current one runs (2 x 2 x 64 for S, 2 x 128 for O).
+    static constexpr int kSBufs = kWide ? 2 : 1;
+    // MMA-issuing warps.  One thread issuing for both streams is enough with 64 channels (two CTAs per SM
+    // share the tensor pipe).  With 128 channels a stream's tile is 12 instructions of 50-65 clocks of issue
+    // each plus three barrier waits, and a single issuer for both streams was what bound the kernel: each
+    // stream gets its own issuing warp (one CTA per SM, so the registers are there).
+    static constexpr int kMmaWarps = kWide ? 2 : 1;
+    static constexpr int kThreads = (kMmaWarp + kMmaWarps) * 32;
+    static constexpr uint32_t kTmemCols = kWide ? 512 : 256;
+    static constexpr uint32_t kSCol = 0, kOCol = 2 * kSBufs * kKT;
+    static constexpr int kCtasPerSm = kWide ? 1 : 2;
 };
 
 constexpr int kTileTab = 256;     // tiles whose (first token, valid tokens) are tabulated in shared memory
@@ -65,7 +79,8 @@ constexpr int kTileTab = 256;     // tiles whose (first token, valid tokens) are
 struct Barriers {
     uint64_t q_full[2][2];     // [stream][half]: see kQSplitRows
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2][2], p_full[2][2];   // [stream][S buffer]
+    uint64_t o_full[2], pv_done[2];
     uint32_t tmem_base;
     int abort_flag;
     int2 tile_tab[kTileTab];
@@ -424,8 +439,8 @@ __device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0,
 }
 
 // ---------------------------------------------------------------- kernel
-template <int D, bool kExt>
-__global__ void __launch_bounds__(kThreads, Cfg<D>::kCtasPerSm)
+template <int D, bool kExt, bool kWide>
+__global__ void __launch_bounds__(Cfg<D, kWide>::kThreads, Cfg<D, kWide>::kCtasPerSm)
 attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap k_map64,
                    const __grid_constant__ CUtensorMap v_map64, const __grid_constant__ ExtArgs ext,
@@ -434,7 +449,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                    const PairPlan pp, int32_t n_tiles, int3 qpos, float scale_log2, int* __restrict__ status)
 {
     const int ext_range = kExt ? ext.range : -1;
-    using C = Cfg<D>;
+    using C = Cfg<D, kWide>;
     extern __shared__ uint8_t smem_raw[];
     Barriers* bars = reinterpret_cast<Barriers*>(smem_raw);
     volatile int* abort_flag = &bars->abort_flag;
@@ -452,18 +467,21 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (int g = 0; g < 2; ++g) {
             mbar_init(smem_u32(&bars->q_full[g][0]), 1);
             mbar_init(smem_u32(&bars->q_full[g][1]), 1);
-            mbar_init(smem_u32(&bars->s_full[g]), 1);
-            mbar_init(smem_u32(&bars->p_full[g]), kGroupWarps);
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(smem_u32(&bars->s_full[g][b]), 1);
+                mbar_init(smem_u32(&bars->p_full[g][b]), kGroupWarps);
+            }
+            mbar_init(smem_u32(&bars->pv_done[g]), 1);
             mbar_init(smem_u32(&bars->o_full[g]), 1);
         }
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars->kv_full[s]), 1);
-            mbar_init(smem_u32(&bars->kv_empty[s]), 1);
+            mbar_init(smem_u32(&bars->kv_empty[s]), C::kMmaWarps);   // one arrival per issuing warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (!layout_ok) report(status, kStatusSyncTimeout, abort_flag);
     }
-    for (int j = threadIdx.x; j < n_tiles && j < kTileTab; j += kThreads) {
+    for (int j = threadIdx.x; j < n_tiles && j < kTileTab; j += C::kThreads) {
         int32_t t0, valid;
         tile_at(ranges, j, t0, valid, ext_range);
         bars->tile_tab[j] = make_int2(t0, valid);
@@ -471,7 +489,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     if (layout_ok) {
         // query rows a tile does not cover keep whatever the slot held before; start them at zero
         uint4* qz = reinterpret_cast<uint4*>(smem_raw + (q_smem - raw));
-        for (uint32_t i = threadIdx.x; i < 2 * C::kQBytes / 16; i += kThreads) qz[i] = make_uint4(0, 0, 0, 0);
+        for (uint32_t i = threadIdx.x; i < 2 * C::kQBytes / 16; i += C::kThreads) qz[i] = make_uint4(0, 0, 0, 0);
         fence_async_smem();
     }
     if (warp == kProducerWarp) {
@@ -500,7 +518,12 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     // rows from wherever the tile starts; what it reads past the tile only reaches dead rows of S.
     const bool q_split = T <= kQSplitRows;
     constexpr uint32_t kQHalfSlot = kQSplitRows * 128;   // bytes from the first to the second tile of a slot
-    const uint32_t s_full0 = smem_u32(&bars->s_full[0]), p_full0 = smem_u32(&bars->p_full[0]);
+    const uint32_t s_full0 = smem_u32(&bars->s_full[0][0]), p_full0 = smem_u32(&bars->p_full[0][0]);   // + 16 g + 8 buffer
+    const uint32_t pv_done0 = smem_u32(&bars->pv_done[0]);
+    // S buffer and barrier phase of a stream's flat tile index: with two buffers they alternate, and each
+    // buffer's barriers see every other tile
+    auto buf_of = [](uint32_t t) -> uint32_t { return C::kSBufs == 2 ? (t & 1u) : 0u; };
+    auto par_of = [](uint32_t t) -> uint32_t { return C::kSBufs == 2 ? ((t >> 1) & 1u) : (t & 1u); };
     const uint32_t o_full0 = smem_u32(&bars->o_full[0]);
     const uint32_t kv_full0 = smem_u32(&bars->kv_full[0]), kv_empty0 = smem_u32(&bars->kv_empty[0]);
 
@@ -643,8 +666,13 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     if (mbar_try_wait(kv_full0 + 8 * stage, use & 1u)) break;
             }
         }
-    } else if (layout_ok && warp == kMmaWarp) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (layout_ok && warp >= kMmaWarp) {
+        // ------------------------------------------------------------ MMA issuer(s)
+        // With two issuing warps, warp kMmaWarp + g issues for stream g only; both walk the same loop, so the
+        // stage counter advances alike in both.  A commit covers the issuing thread's own instructions only,
+        // hence a key/value stage is released by one arrival per issuing warp: each commits its own P V on a
+        // shared tile, and the one stream that uses a tile of its own commits twice.
+        const int my_g = C::kMmaWarps == 2 ? warp - kMmaWarp : -1;   // -1: this warp issues for both streams
         if (my_pairs > 0) {
             bool ok = true;
             const uint32_t idesc_pv = make_idesc(kQRows, D, 1);
@@ -653,9 +681,9 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             const uint32_t q_lo0 = desc_lo(q_smem, 16);
             constexpr uint32_t kStageLo = C::kStageBytes >> 4, kQLo = C::kQBytes >> 4;
             // per stream: the tile whose S was issued last and whose P V is still to be issued
-            uint32_t pv_stage[2] = {0, 0}, pv_nch[2] = {0, 0};
+            uint32_t pv_stage[2] = {0, 0}, pv_nch[2] = {0, 0}, pv_t[2] = {0, 0};
             bool pv_live[2] = {false, false}, pv_first[2] = {false, false}, pv_release[2] = {false, false},
-                 pv_last[2] = {false, false};
+                 pv_last[2] = {false, false}, pv_twice[2] = {false, false};
             uint32_t tcount[2] = {0, 0};   // tiles issued per stream
             uint32_t ucount[2] = {0, 0};   // units started per stream
             uint32_t q_half[2] = {0, 0};   // half of the query slot the current unit of each stream uses
@@ -664,13 +692,13 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             // O (+)= P V : M = 128, N = D channels, K = 16 * nch tokens; P from TMEM (packed over S),
             // V read MN-major from its stage
             auto issue_pv = [&](const int g) -> bool {
-                const uint32_t t = tcount[g] - 1;  // flat tile index of this stream
-                if (!warp_wait(p_full0 + 8 * g, t & 1u, abort_flag)) return false;
+                const uint32_t t = pv_t[g];  // flat tile index of this stream
+                if (!warp_wait(p_full0 + 16 * g + 8 * buf_of(t), par_of(t), abort_flag)) return false;
                 // (a unit's first P V overwrites O: every warp of the group arrives on p_full for that tile
                 // only after its epilogue of the previous unit, so O has been read by then)
                 tc_fence_after();
                 const uint32_t v_lo = v_lo0 + pv_stage[g] * kStageLo;
-                const uint32_t p_tmem = tmem + C::kSCol + g * kKT;
+                const uint32_t p_tmem = tmem + C::kSCol + (g * C::kSBufs + buf_of(t)) * kKT;
                 const uint32_t o_tmem = tmem + C::kOCol + g * D;
                 const uint32_t nch = pv_nch[g];
                 if (elect_one()) {
@@ -679,7 +707,9 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     if (nch > 2) umma_ts(o_tmem, p_tmem + 16, v_lo + (4096 >> 4), kDescHi, idesc_pv, 1u);
                     if (nch > 3) umma_ts(o_tmem, p_tmem + 24, v_lo + (6144 >> 4), kDescHi, idesc_pv, 1u);
                     if (pv_release[g]) umma_commit(kv_empty0 + 8 * pv_stage[g]);
+                    if (C::kMmaWarps == 2 && pv_twice[g]) umma_commit(kv_empty0 + 8 * pv_stage[g]);
                     if (pv_last[g]) umma_commit(o_full0 + 8 * g);
+                    if (C::kSBufs == 2) umma_commit(pv_done0 + 8 * g);   // read by the (rare) rescale of O only
                 }
                 __syncwarp();
                 return true;
@@ -697,6 +727,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
                         if (!ok) continue;
+                        if (my_g >= 0 && g != my_g) continue;
                         if (g >= ng) {
                             // the stream is absent from this pair: its last P V of the previous pair must not
                             // wait for a next S that is not coming soon (it also holds a key/value stage)
@@ -717,14 +748,20 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                             if (!warp_wait(q_full0 + 16 * g + 8 * q_half[g], parity, abort_flag)) { ok = false; continue; }
                             ++ucount[g];
                         }
-                        if (!(shared && g == 1)) {  // the second stream of a shared tile finds it landed already
+                        if (!(shared && g == 1 && my_g < 0)) {  // one issuer: the second stream of a shared tile finds it landed
                             if (!warp_wait(kv_full0 + 8 * stage, use & 1u, abort_flag)) { ok = false; continue; }
                         }
-                        if (pv_live[g] && !issue_pv(g)) { ok = false; continue; }
+                        // One S buffer: the pending P V of the previous tile goes first, because this S
+                        // overwrites its P.  Two buffers: this S goes first and runs on the tensor pipe while
+                        // the softmax of the previous tile finishes (streams with tiles of their own keep the
+                        // first order: they need their key/value stages back sooner).
+                        const bool s_first = C::kSBufs == 2 && shared;
+                        if (!s_first && pv_live[g] && !issue_pv(g)) { ok = false; continue; }
                         tc_fence_after();
+                        const uint32_t t_now = tcount[g];
                         const uint32_t q_lo = q_lo0 + g * kQLo + q_half[g] * (kQHalfSlot >> 4);
                         const uint32_t k_lo = k_lo0 + stage * kStageLo;
-                        const uint32_t d = tmem + C::kSCol + g * kKT;
+                        const uint32_t d = tmem + C::kSCol + (g * C::kSBufs + buf_of(t_now)) * kKT;
                         if (elect_one()) {
                             umma_ss<false>(d, q_lo, k_lo, kDescHi, idesc_s);
 #pragma unroll
@@ -733,15 +770,18 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                                 umma_ss<true>(d, q_lo + (ks >> 2) * kQH + (ks & 3) * 2,
                                               k_lo + (ks >> 2) * kKH + (ks & 3) * 2, kDescHi, idesc_s);
                             }
-                            umma_commit(s_full0 + 8 * g);
+                            umma_commit(s_full0 + 16 * g + 8 * buf_of(t_now));
                         }
                         __syncwarp();
+                        if (s_first && pv_live[g] && !issue_pv(g)) { ok = false; continue; }
                         pv_live[g] = true;
                         pv_stage[g] = stage;
                         pv_nch[g] = nch;
+                        pv_t[g] = t_now;
                         pv_first[g] = (j == 0);
                         pv_last[g] = (j == n_tiles - 1);
-                        pv_release[g] = shared ? (g == ng - 1) : true;
+                        pv_release[g] = (shared && my_g < 0) ? (g == ng - 1) : true;
+                        pv_twice[g] = !shared;
                         ++tcount[g];
                     }
                     sq += shared ? 1 : ng;
@@ -749,7 +789,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
 #pragma unroll
             for (int g = 0; g < 2; ++g)
-                if (ok && pv_live[g] && !issue_pv(g)) ok = false;
+                if (ok && (my_g < 0 || g == my_g) && pv_live[g] && !issue_pv(g)) ok = false;
             if (!ok && lane == 0) report(status, kStatusMmaTimeout, abort_flag);
         }
     } else if (layout_ok) {
@@ -757,9 +797,8 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int g = warp >> 2, wq = warp & 3;
         const uint32_t lane_base = ((uint32_t)(wq * 32)) << 16;
         const int r = wq * 32 + lane;  // query row inside the tile = TMEM lane
-        const uint32_t s_tmem = tmem + C::kSCol + g * kKT + lane_base;
+        const uint32_t s_tmem0 = tmem + C::kSCol + g * C::kSBufs * kKT + lane_base;   // + kKT per S buffer
         const uint32_t o_tmem = tmem + C::kOCol + g * D + lane_base;
-        const uint32_t s_full = s_full0 + 8 * g, p_full = p_full0 + 8 * g;
         const uint32_t o_full = o_full0 + 8 * g;
         const bool q_loader = (wq == 0 && lane == 0);
         uint32_t q_armed = 0;     // query tiles requested so far
@@ -810,7 +849,9 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             for (int j = 0; j < n_tiles; ++j, ++t) {
                 int32_t t0, valid;
                 tile_of(j, t0, valid);
-                if (!__all_sync(0xffffffffu, mbar_wait(s_full, t & 1u, abort_flag))) {
+                const uint32_t s_tmem = s_tmem0 + buf_of(t) * kKT;
+                const uint32_t s_full = s_full0 + 16 * g + 8 * buf_of(t), p_full = p_full0 + 16 * g + 8 * buf_of(t);
+                if (!__all_sync(0xffffffffu, mbar_wait(s_full, par_of(t), abort_flag))) {
                     report(status, kStatusSyncTimeout, abort_flag);
                     ok = false;
                     break;
@@ -846,8 +887,17 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     } else {
                         const bool grow = fmaf(mt, scale_log2, nb) > kRescaleLog2;
                         if (__any_sync(0xffffffffu, grow)) {
-                            // rare: bring O and the row sum to the new reference.  The previous P V is done:
-                            // it was issued before this tile's S, whose arrival covers every earlier product.
+                            // rare: bring O and the row sum to the new reference.  The previous P V must be done.
+                            // One S buffer: it was issued before this tile's S, whose arrival covers every
+                            // earlier product.  Two buffers: this S may have been issued first, so wait for the
+                            // product's own completion (one arrival per P V; at most one phase can be ahead,
+                            // because the next P V needs the P this tile has not written yet).
+                            if (C::kSBufs == 2 && !__all_sync(0xffffffffu, mbar_wait(pv_done0 + 8 * g, (t - 1u) & 1u, abort_flag))) {
+                                report(status, kStatusSyncTimeout, abort_flag);
+                                ok = false;
+                                break;
+                            }
+                            if (C::kSBufs == 2) tc_fence_after();
                             float alpha = 1.f;
                             if (grow) {
                                 alpha = fast_exp2((m_ref - mt) * scale_log2);
@@ -950,19 +1000,19 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 }
 
 // ---------------------------------------------------------------- host side
-template <int D, bool kExt>
+template <int D, bool kExt, bool kWide>
 cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& km64,
                    const CUtensorMap& vm64, const ExtArgs& ext, const Strided& O,
                    const RangeList& ranges, int32_t T, int32_t heads, const PairPlan& pp, int32_t n_tiles, int3 qpos,
                    float scale_log2, int* status, int sm_count, cudaStream_t stream)
 {
-    using C = Cfg<D>;
+    using C = Cfg<D, kWide>;
     static SharedMemoryOptIn opt_in;
-    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt>, (int)C::kSmemBytes);
+    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide>, (int)C::kSmemBytes);
     if (oe != cudaSuccess) return oe;
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > pp.n_pairs) grid = pp.n_pairs;
-    attend_pair_kernel<D, kExt><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(
+    attend_pair_kernel<D, kExt, kWide><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
         qm, km, vm, km64, vm64, ext, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos,
         scale_log2, status);
     count_launch();
@@ -1020,18 +1070,19 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     for (int i = 0; i < ranges.n; ++i) n_tiles += (ranges.r[i].len + kKT - 1) / kKT;
     const int3 qpos = make_int3(pos[0], pos[1], pos[2]);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
-    if (cur) {
-        if (D == 64)
-            return launch<64, true>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
-                                    sm_count, stream);
-        return launch<128, true>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
-                                 sm_count, stream);
+    // 64 channels always take the two-CTA form: the wide form was measured on the tensor-bound launches of a
+    // 2 240-token schedule (T = 576 and 1 024, 36 heads) and lost there too (26.3 vs 20.8 and 64.2 vs 53.9 ms):
+    // two streams per SM do not keep the tensor pipe as busy as four, even with the chain broken.
+#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE)                                                                             \
+    return launch<DD, EXT, WIDE>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status, \
+                                 sm_count, stream)
+    if (D == 128) {
+        if (cur) AMSKV_PAIR_LAUNCH(128, true, true);
+        AMSKV_PAIR_LAUNCH(128, false, true);
     }
-    if (D == 64)
-        return launch<64, false>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
-                                 sm_count, stream);
-    return launch<128, false>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status,
-                              sm_count, stream);
+    if (cur) AMSKV_PAIR_LAUNCH(64, true, false);
+    AMSKV_PAIR_LAUNCH(64, false, false);
+#undef AMSKV_PAIR_LAUNCH
 }
 
 }  // namespace amskv

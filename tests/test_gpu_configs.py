@@ -26,7 +26,7 @@ def _query_rows(T, g, n=96):
     return sorted(fixed | set(rnd))[: n + len(fixed)]
 
 
-def _check_sampled(wl, pols, n_items, seed, path=B.PATH_AUTO, need_gb=4.0):
+def _check_sampled(wl, pols, n_items, seed, path=B.PATH_AUTO, need_gb=4.0, fused=False):
     free_b, _ = torch.cuda.mem_get_info()
     if free_b < need_gb * 1e9:
         pytest.skip("needs about %.0f GB of device memory" % need_gb)
@@ -43,7 +43,7 @@ def _check_sampled(wl, pols, n_items, seed, path=B.PATH_AUTO, need_gb=4.0):
 
     scale = 1.0 / math.sqrt(wl.head_dim)
     with Cache(len(pols), wl.heads, wl.head_dim, wl.rows, wl.sides, pols) as cache:
-        outs = run_pass(cache, qkv, path)
+        outs = run_pass(cache, qkv, path, fused=fused)
         Ks = [pick(k).cpu().double().numpy() for _, k, _ in qkv]
         Vs = [pick(v).cpu().double().numpy() for _, _, v in qkv]
         for k, (q, _, _) in enumerate(qkv):
@@ -71,11 +71,14 @@ def test_text_to_image_1024_shape_sampled():
     _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 3, seed=12, need_gb=3.0)
 
 
-def test_depth_36_512_shape_sampled():
+@pytest.mark.parametrize("fused", [False, True], ids=["separate", "fused"])
+def test_depth_36_512_shape_sampled(fused):
     """36 heads x 64 (dim 2304), ten scales up to 32 x 32 (2 240 tokens): head_dim 64 with eight query
-    tiles per item at the last scale, one layer of each class, sampled items and query rows."""
+    tiles per item at the last scale (the tensor-bound launches take the one-CTA-per-SM form of the paired
+    kernel), one layer of each class, sampled items and query rows."""
     wl = synth.WORKLOADS["var_d36_512"].replace(batch=8)
-    _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 6, seed=14, need_gb=3.0)
+    _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 6, seed=14, need_gb=3.0,
+                   fused=fused)
 
 
 @pytest.mark.parametrize("batch", [1, 16])
