@@ -99,6 +99,7 @@ struct PairPlan {
     int32_t n_items;
     int32_t n_shared;     // = n_items * npi
     int32_t n_pairs;      // n_shared + ceil(n_items * (nqt & 1) / 2)
+    int32_t kind;         // 0: no pair is shared, 1: every pair is, 2: both kinds (so that the common cases test a launch constant)
 };
 
 // The current scale read from the caller's K/V tensors instead of the cache: the last entry of the
@@ -120,12 +121,15 @@ struct Stream {
     bool valid;
 };
 
-__device__ __forceinline__ bool pair_is_shared(const PairPlan& pp, int32_t pair) { return pair < pp.n_shared; }
+__device__ __forceinline__ bool pair_is_shared(const PairPlan& pp, int32_t pair)
+{
+    return pp.kind == 2 ? pair < pp.n_shared : pp.kind == 1;
+}
 
 __device__ __forceinline__ Stream stream_of(const PairPlan& pp, int32_t pair, int g)
 {
     Stream s;
-    if (pair < pp.n_shared) {
+    if (pair_is_shared(pp, pair)) {
         s.item = pp.npi == 1 ? pair : pair / pp.npi;
         s.qt = 2 * (pair - s.item * pp.npi) + g;
         s.valid = true;
@@ -1066,6 +1070,7 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     if (n_pairs > 0x7fffffffll) return cudaErrorInvalidValue;
     pp.n_shared = (int32_t)n_shared;
     pp.n_pairs = (int32_t)n_pairs;
+    pp.kind = pp.npi == 0 ? 0 : ((pp.nqt & 1) ? 2 : 1);
     int32_t n_tiles = 0;
     for (int i = 0; i < ranges.n; ++i) n_tiles += (ranges.r[i].len + kKT - 1) / kKT;
     const int3 qpos = make_int3(pos[0], pos[1], pos[2]);
