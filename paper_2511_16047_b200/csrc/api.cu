@@ -395,11 +395,31 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
         ranges.n = lay.ranges_before(cache->tokens, scale, ranges.r);
         if (ranges.n >= kMaxRanges) fused = false;
     }
+    int32_t rider_tok = 0, rider_valid = 0;
+    if (fused) {
+        // The kernel works in 64-token key tiles per range.  Up to 16 tokens left over at the end of a cache
+        // range (the condensed scales behind a 64-token scale, say) would cost a tile of their own; when the
+        // current scale's last tile has a 16-token box to spare they ride there instead.
+        const int32_t tail = T % 64;
+        if (tail >= 1 && tail <= 48) {
+            for (int i = ranges.n - 1; i >= 0 && rider_valid == 0; --i) {
+                const int32_t left = ranges.r[i].len % 64;
+                if (left >= 1 && left <= 16) {
+                    rider_valid = left;
+                    rider_tok = ranges.r[i].start + ranges.r[i].len - left;
+                    ranges.r[i].len -= left;
+                    if (ranges.r[i].len == 0) {
+                        for (int m = i; m + 1 < ranges.n; ++m) ranges.r[m] = ranges.r[m + 1];
+                        --ranges.n;
+                    }
+                }
+            }
+        }
+    }
     if (fused && cache->path == AMSKV_PATH_AUTO) {
-        // The kernel works in 64-token key tiles per range.  Taking the scale from the caller's tensors
-        // splits it off the range it would be part of in the cache; where that adds a tile, attention
-        // loses more than the saved copy is worth (measured), so such scales run as the two calls
-        // (AMSKV_PATH_TENSOR_PAIR fuses wherever it can).
+        // Taking the scale from the caller's tensors splits it off the range it would be part of in the
+        // cache; where that adds a tile, attention loses more than the saved copy is worth (measured), so
+        // such scales run as the two calls (AMSKV_PATH_TENSOR_PAIR fuses wherever it can).
         auto tiles = [](const RangeList& rl) {
             int32_t n = 0;
             for (int i = 0; i < rl.n; ++i) n += (rl.r[i].len + 63) / 64;
@@ -419,6 +439,8 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
     ranges.total = 0;
     for (int i = 0; i < ranges.n; ++i) ranges.total += ranges.r[i].len;
     CurrentScaleSource cur{ks, vs, true, piece[0].dst, cache->region(layer)};
+    cur.rider_tok = rider_tok;
+    cur.rider_valid = rider_valid;
     cudaError_t e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes,
                                        cache->k_maps64[layer].bytes, cache->v_maps64[layer].bytes, ranges, T, cache->rows,
                                        cache->heads, cache->head_dim, cache->softmax_scale, cache->status_word(),

@@ -113,6 +113,7 @@ struct ExtArgs {
     int32_t store;
     int32_t dst;                      // first position of the scale in the per-item region
     int3 pos;                         // coordinate slots of token, head and row in the rank-4 maps
+    int32_t rider_tok, rider_valid;   // older cache tokens that ride in the spare box of the scale's last tile
 };
 
 struct Stream {
@@ -578,6 +579,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 const bool from_ext = kExt && (t0 & kExtFlag) != 0;
                 t0 &= ~kExtFlag;
                 const int nch = (valid + 15) >> 4;
+                const bool rider = kExt && ext.rider_valid > 0 && j == n_tiles - 1;   // one more box, from the cache
                 for (int g = 0; g < per_tile; ++g, ++sq) {
                     const int item = g == 0 ? sa.item : sb.item;
                     const uint32_t stage = sq % C::kStages, use = sq / C::kStages;
@@ -599,7 +601,16 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     const uint32_t full = kv_full0 + 8 * stage;
                     const uint32_t k_dst = kv_smem + stage * C::kStageBytes, v_dst = k_dst + C::kKVBytes;
                     if (elect_one()) {
-                        mbar_expect_tx(full, (uint32_t)nch * kKVBoxRows * D * 2 * 2);
+                        mbar_expect_tx(full, (uint32_t)(nch + (rider ? 1 : 0)) * kKVBoxRows * D * 2 * 2);
+                        if (rider) {
+#pragma unroll
+                            for (int h = 0; h < C::kHalves; ++h) {
+                                tma_load_3d(k_dst + h * C::kKVHalfBytes + nch * kKVBoxRows * 128, &k_map, full, h * 64,
+                                            ext.rider_tok, item);
+                                tma_load_3d(v_dst + h * C::kKVHalfBytes + nch * kKVBoxRows * 128, &v_map, full, h * 64,
+                                            ext.rider_tok, item);
+                            }
+                        }
                         if (from_ext) {
                             const int32_t row = item / heads, head = item - row * heads;
                             int c[4] = {0, 0, 0, 0};
@@ -726,7 +737,8 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     int32_t t0, valid;
                     tile_of(j, t0, valid);
-                    const uint32_t nch = (uint32_t)(valid + 15) >> 4;
+                    const uint32_t nch = ((uint32_t)(valid + 15) >> 4) +
+                                         ((kExt && ext.rider_valid > 0 && j == n_tiles - 1) ? 1u : 0u);
                     const uint32_t idesc_s = make_idesc(kQRows, nch * 16, 0);
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
@@ -867,9 +879,15 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     uint32_t sr[kKT];
                     tmem_ld64(s_tmem, sr);
                     if (valid < kKT) {
+                        // (a rider occupies the box behind the tile's own: its tokens stay, the gap before them goes)
+                        // as a bit per column, so that each column costs one test of a constant bit
+                        uint64_t keep = (1ull << valid) - 1ull;
+                        if (kExt && ext.rider_valid > 0 && j == n_tiles - 1)
+                            keep |= ((1ull << ext.rider_valid) - 1ull) << ((valid + 15) & ~15);
+                        const uint32_t keep_lo = (uint32_t)keep, keep_hi = (uint32_t)(keep >> 32);
 #pragma unroll
                         for (int i = 0; i < kKT; ++i)
-                            if (i >= valid) sr[i] = 0xff800000u;  // -inf
+                            if ((((i < 32 ? keep_lo : keep_hi) >> (i & 31)) & 1u) == 0u) sr[i] = 0xff800000u;  // -inf
                     }
                     // row maximum with four independent chains
                     float mx[4];
@@ -1048,6 +1066,12 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
         ext.range = ranges.n - 1;
         ext.store = cur->store ? 1 : 0;
         ext.dst = cur->dst;
+        if (cur->rider_valid > 0) {
+            const int32_t tail = T % kKT;
+            if (cur->rider_valid > kKVBoxRows || tail < 1 || tail > kKT - kKVBoxRows) return cudaErrorInvalidValue;
+            ext.rider_tok = cur->rider_tok;
+            ext.rider_valid = cur->rider_valid;
+        }
         if (cur->store &&
             !tc_encode_kv_store_maps(cur->region, (int64_t)rows * heads, D, kKT, cur->dst + T, &ext.k_store, &ext.v_store))
             return cudaErrorNotSupported;

@@ -49,11 +49,16 @@ cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion&
 // The current scale taken from the caller's K/V tensors instead of the cache: the last entry of the
 // range list given with it stands for that scale (start 0, len T).  With `store`, the kernel also
 // writes the scale to position `dst` of every item's part of `region` (the append fused into attention).
+// `rider`: up to 16 older tokens of the cache (positions rider_tok .. rider_tok + rider_valid - 1) that are
+// not in the range list but ride in the free 16-token box of the scale's last, partly filled key tile, so
+// that they do not cost a tile of their own (rider_valid = 0: none; the scale's last tile must then have
+// a box to spare: (T mod 64) in 1..48).
 struct CurrentScaleSource {
     Strided K, V;
     bool store;
     int32_t dst;
     LayerRegion region;
+    int32_t rider_tok = 0, rider_valid = 0;
 };
 
 // (the CUDA-core kernel takes a current-scale source without `store` only)

@@ -75,6 +75,25 @@ def test_ragged_tiles_many_items_and_strided_inputs(D):
                 check_close(outs[layer][k], want[k], "D %d layer %d scale %d" % (D, layer, k))
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_left_over_cache_tokens_ride_in_the_spare_box_of_the_last_tile(D):
+    """5 condensed tokens behind a 64-token scale would be a key tile of their own; with a 100-token current
+    scale (last tile 36 tokens) they are loaded into that tile's fourth 16-token box instead.  Also a
+    one-token and a 16-token remainder, and an odd number of items (a unit with a single stream)."""
+    _need(D)
+    for sides, pols in [((1, 2, 8, 10), [(2, 2, False)]), ((1, 6), [(1, 1, False), (2, 2, True)]), ((4, 8, 5), [(1, 2, False)])]:
+        rows, heads = 3, 5
+        qkv = make_qkv(rows, heads, sides, D, seed=46 + len(sides))
+        scale = 1.0 / math.sqrt(D)
+        for path in (B.PATH_AUTO, B.PATH_TENSOR_PAIR):
+            with Cache(len(pols), heads, D, rows, sides, pols) as c:
+                outs = run_pass(c, qkv, path, fused=True)
+                for layer, pol in enumerate(pols):
+                    want = oracle_outputs(qkv, pol, scale)
+                    for k in range(len(sides)):
+                        check_close(outs[layer][k], want[k], "sides %s layer %d scale %d" % (sides, layer, k))
+
+
 def test_token_budgets_fused():
     """Under token budgets the fused path takes the appends that are one copy; the rest run as two calls."""
     _need()
