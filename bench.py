@@ -35,7 +35,7 @@ FALLBACK_BF16_TFLOPS = 1400.0
 # dram__bytes_write.sum of every launch of those calls in a 64-row case, scaled by rows and layers; the
 # capture is summarised under profiles/), keyed by (workload, policy, calls).  Only valid for the
 # default batch and layer count and for the kernels as they were when it was captured.
-NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams", "fused"): 278.7e9}
+NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams", "fused"): 273.5e9}
 
 
 def _peaks():
