@@ -180,7 +180,8 @@ AMSKV_API int amskv_append(amskv_cache* cache, int layer, int scale, const void*
  * (Sec. 3.1, Eq. 2: a whole scale is conditioned on whole earlier scales, so there is no
  * mask inside the retained set):  out = softmax(softmax_scale * Q K^T) V.
  *   Q, out    device pointers, [rows, heads, T, head_dim] bf16; strides as in append.
- * `scale` must be the scale most recently appended to `layer` (ORDER otherwise).
+ * `scale` must be the scale most recently appended to `layer` (ORDER otherwise).  out must not
+ * overlap Q.
  * Arithmetic: bf16 inputs, fp32 accumulation, probabilities rounded to bf16 before the
  * second product on the tensor-core path, bf16 output.
  */
@@ -199,7 +200,7 @@ AMSKV_API int amskv_attend(amskv_cache* cache, int layer, int scale, const void*
  * scales of fewer than 64 tokens and scales where splitting the current scale off its cache range
  * would add a 64-token key tile, run as the two calls.
  *   K, V: as for amskv_append (one stride triple kv_strides for both); Q, out: as for
- *   amskv_attend.  out must not alias K or V.
+ *   amskv_attend.  out must not overlap Q, K or V.
  * Stream ordering: as for the two calls -- this call must come after attend(layer, scale - 1)
  * has finished reading (same stream, or an event).
  */
