@@ -31,11 +31,11 @@ UNIT = "us/image"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0
 
-# DRAM traffic of the timed calls per step, from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of every launch of those calls in a 64-row case, scaled by rows and layers; the
-# capture is summarised under profiles/), keyed by (workload, policy, calls).  Only valid for the
-# default batch and layer count and for the kernels as they were when it was captured.
-NCU_TRAFFIC_BYTES_PER_STEP = {("var_d30", "ams", "fused"): 273.5e9}
+# DRAM traffic of the dominant kernel per launch, from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by (workload, policy, calls); each entry names the capture it came from and
+# is valid only for the kernel as it was then -- an entry is removed whenever that kernel changes, and
+# `roofline.traffic` is then null.
+NCU_DOMINANT_KERNEL_TRAFFIC = {}
 
 
 def _peaks():
@@ -154,10 +154,15 @@ def run_ours(args):
     tok = wl.tokens
     stream = torch.cuda.current_stream()
 
-    # inputs: one Q/K/V set per scale, shared by the layers (each layer has its own cache region,
-    # so no K/V read by attention is shared between layers)
-    qkv = [synth.qkv_for_scale(wl.rows, wl.heads, tok[k], wl.head_dim, wl.seed, k, "cuda") for k in range(K)]
-    outs = [torch.empty_like(q) for q, _, _ in qkv]
+    # inputs: several Q/K/V sets per scale, used by the layers in turn.  Each layer has its own cache region,
+    # so no cached K/V is shared between layers; the scale's own Q/K/V are inputs, and with one set a layer
+    # could find the coarse scales' inputs (up to ~140 MB) in the 126 MB L2 where the previous layer left
+    # them.  With the sets rotating, a set is touched again only after the others' bytes went through L2.
+    n_sets = max(1, args.input_sets)
+    qkv_sets = [[synth.qkv_for_scale(wl.rows, wl.heads, tok[k], wl.head_dim, wl.seed + 101 * i, k, "cuda") for k in range(K)]
+                for i in range(n_sets)]
+    qkv = qkv_sets[0]
+    outs_sets = [[torch.empty_like(q) for q, _, _ in qs] for qs in qkv_sets]
     input_bytes = sum(3 * q.numel() * 2 for q, _, _ in qkv)
 
     def measure(policies, label, instrument, streams=None, budgets=None, fuse=None):
@@ -193,8 +198,9 @@ def run_ours(args):
             if side is not None:
                 side.wait_stream(stream)
             for k in range(K):
-                q, kk, v = qkv[k]
                 for layer in range(wl.layers):
+                    q, kk, v = qkv_sets[layer % n_sets][k]
+                    out = outs_sets[layer % n_sets][k]
                     i = k * wl.layers + layer
                     if side is not None:
                         if k > 0:
@@ -209,10 +215,10 @@ def run_ours(args):
                         e0.record(stream)
                     if fuse:
                         n0 = B.amskv_launch_count()
-                        B.amskv_append_attend(cache, layer, k, kk, v, q, outs[k], stream)
+                        B.amskv_append_attend(cache, layer, k, kk, v, q, out, stream)
                         fused_launch[(layer, k)] = B.amskv_launch_count() - n0 == 1
                     else:
-                        B.amskv_attend(cache, layer, k, q, outs[k], stream)
+                        B.amskv_attend(cache, layer, k, q, out, stream)
                     if events is not None:
                         e1.record(stream)
                     if side is not None:
@@ -256,15 +262,24 @@ def run_ours(args):
         ms = t0.elapsed_time(t1)
         result = {"label": label, "ms_per_step": ms / args.steps, "launches_per_step": launches_per_step,
                   "kv_bytes": B.amskv_cache_bytes(cache)[2], "arena_bytes": nbytes, "fused": bool(fuse)}
+        # Minimum bytes of a step: Q read + out written + the kept K/V read once (`work`), plus the scale's own
+        # K/V written to the cache once.  A call that ran as copy kernel + attention also reads the scale's K/V
+        # a second time (the copy reads them, attention reads them again from the cache): counted apart, as
+        # wasted bytes, never as work.  With --no-fuse the timed calls are the attention launches alone.
+        items = wl.rows * wl.heads
+        wasted = {key: 0 for key in work}
+        one_launch = {key: False for key in work}
         if fuse:
-            # the timed calls now carry the append as well: the K/V of the scale written once by the fused
-            # launch (read once either way); where the call ran as two launches, also read by the copy
-            items = wl.rows * wl.heads
             for (layer, k), (b, f) in list(work.items()):
                 kv = 2 * wl.head_dim * items * 2 * tok[k]
                 if args.transient_last and k == K - 1:
                     kv = 0   # attended from the caller's tensors, never written
-                work[(layer, k)] = (b + (kv if fused_launch.get((layer, k)) else 2 * kv), f)
+                work[(layer, k)] = (b + kv, f)
+                one_launch[(layer, k)] = bool(fused_launch.get((layer, k)))
+                wasted[(layer, k)] = 0 if one_launch[(layer, k)] else kv
+        result["wasted_bytes_per_step"] = sum(wasted.values())
+        result["step_bytes"] = sum(b for b, _ in work.values()) + (
+            0 if fuse else sum(2 * wl.head_dim * items * 2 * tok[k] for (_, k) in work))
 
         if instrument:
             # per-launch durations of the attention kernel: same steps, eager, CUDA events on the launch stream
@@ -296,6 +311,16 @@ def run_ours(args):
                                   "frac": round(roof / t, 3) if t else None})
             result["per_scale"] = per_scale
             result["pass_roofline_ms"] = sum(p["roofline_ms"] for p in per_scale)
+            # the dominant kernel alone: the calls that ran as ONE launch of the paired kernel with the append
+            # fused in (every launch of that kernel in a step, and nothing else, sits between their events)
+            dom = [key for key in work if one_launch[key]]
+            if dom:
+                d_ms = sum(att_ms[key] for key in dom) / args.steps
+                d_bytes = sum(work[key][0] for key in dom)
+                result["dominant"] = {"kernel": "attend_pair_kernel<%d, ext=true, wide=%s>" % (wl.head_dim, "true" if wl.head_dim == 128 else "false"),
+                                      "launches_per_step": len(dom), "bytes_per_step": d_bytes,
+                                      "flops_per_step": sum(work[key][1] for key in dom),
+                                      "ms_per_step": d_ms, "scales": sorted({k for _, k in dom})}
         result["clocks"] = sampler.stop()
         torch.cuda.synchronize()
         assert B.amskv_status(cache) == 0
@@ -400,15 +425,15 @@ def run_ours(args):
         cpu_baseline = oracle_sample(wl, policies, args.cpu_rows, budgets=budgets)
 
     if rank == 0:
-        att_s = main["attend_ms_per_step"] / 1e3
-        achieved = main["attend_bytes_per_step"] / att_s / 1e9
+        # whole pass: minimum bytes of a step over the graph-timed step (launch gaps and all)
+        achieved = main["step_bytes"] / (ms / 1e3) / 1e9
+        dom = main.get("dominant")
         traffic = None
-        if (not args.batch and not args.layers and args.path == "auto" and args.condensed is None and args.local is None
-                and args.demanding_fraction is None):
-            # (the capture is of the configuration named by the key; "fused" = the default calls)
-            per_step = NCU_TRAFFIC_BYTES_PER_STEP.get((args.workload, args.policy, "fused" if main.get("fused") else "separate"))
-            if per_step is not None:
-                traffic = round(per_step / (wl.layers * K))   # per attention launch, like `achieved`
+        if (dom and not args.batch and not args.layers and args.path == "auto" and args.condensed is None
+                and args.local is None and args.demanding_fraction is None):
+            cap = NCU_DOMINANT_KERNEL_TRAFFIC.get((args.workload, args.policy, "fused" if main.get("fused") else "separate"))
+            if cap is not None:
+                traffic = cap
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms, 4), "higher_is_better": False, "scaling": "weak",
@@ -421,7 +446,7 @@ def run_ours(args):
                        "step": "append + attend for every scale and layer",
                        "calls": ("amskv_append_attend (one launch where the paired kernel takes the append in, else two)"
                                  if main.get("fused") else "amskv_append, then amskv_attend"),
-                       "l2": "inputs and per-layer KV regions far larger than L2; no flush needed",
+                       "l2": "per-layer KV regions far larger than L2; %d input sets (Q, K, V, out per scale) used by the layers in turn; no flush" % n_sets,
                        "launch": "CUDA graph replay" if not args.no_graph else "eager",
                        "streams": "appends on a side stream, ordered with attention by events" if args.streams == 2 else "one stream",
                        "last_scale": "never stored" if (args.transient_last and main.get("fused")) else "stored",
@@ -429,12 +454,22 @@ def run_ours(args):
             "clocks": main["clocks"],
             "e2e": e2e,
             "gpu_launches": main["launches_per_step"] * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "attention (all attend launches of a step; with the append fused in where amskv_append_attend does so)" if main.get("fused") else "attention (all attend launches of a step)",
-                         "achieved": round(achieved, 1), "peak": hbm_gbs, "unit": "GB/s",
-                         "frac": round(achieved / hbm_gbs, 4), "peak_kind": peak_kind, "traffic": traffic,
-                         "algorithmic_bytes_per_launch": round(main["attend_bytes_per_step"] / (wl.layers * K)),
-                         "launches_per_step": wl.layers * K,
-                         "frac_of_8TBs_nominal": round(achieved / 8000.0, 4)},
+            "roofline": {"bound": "hbm", "peak": hbm_gbs, "unit": "GB/s", "peak_kind": peak_kind,
+                         "scope": "whole step: minimum bytes (Q read, out written, kept K/V read once, the scale's K/V "
+                                  "written once) / CUDA-graph-timed step",
+                         "achieved": round(achieved, 1), "frac": round(achieved / hbm_gbs, 4),
+                         "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
+                         "step_bytes": main["step_bytes"], "wasted_bytes_per_step": main["wasted_bytes_per_step"],
+                         "wasted_note": "second read of a scale's K/V where a call ran as copy kernel + attention; not counted as work",
+                         "kernel": dom["kernel"] if dom else None,
+                         "kernel_launches_per_step": dom["launches_per_step"] if dom else None,
+                         "kernel_scales": dom["scales"] if dom else None,
+                         "kernel_bytes_per_launch": round(dom["bytes_per_step"] / dom["launches_per_step"]) if dom else None,
+                         "kernel_ms_per_launch": round(dom["ms_per_step"] / dom["launches_per_step"], 5) if dom else None,
+                         "kernel_achieved": round(dom["bytes_per_step"] / dom["ms_per_step"] / 1e6, 1) if dom else None,
+                         "kernel_frac": round(dom["bytes_per_step"] / dom["ms_per_step"] / 1e6 / hbm_gbs, 4) if dom else None,
+                         "kernel_timing": "CUDA events around each call in an eager replay of the same step",
+                         "traffic": traffic},
             "pass_roofline": {"roofline_ms": round(main["pass_roofline_ms"], 3),
                               "attend_ms": round(main["attend_ms_per_step"], 3),
                               "frac": round(main["pass_roofline_ms"] / main["attend_ms_per_step"], 4),
@@ -522,6 +557,7 @@ def oracle_sample(wl, policies, rows, flop_budget=1.0e12, budgets=None):
     images = rows / 2.0
     head_scale = wl.heads / float(heads)
     return {"value": round(weighted * head_scale * 1e6 / images, 1), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "extrapolated": True,
             "sample": "%d rows x %d of %d heads, one layer of each policy kind (%d kinds), all %d scales: %.1f s measured; "
                       "value = extrapolation (linear in rows, heads, layers) to %d heads and %d layers" % (
                           rows, heads, wl.heads, len(kinds), K, total_s, wl.heads, wl.layers),
@@ -556,7 +592,9 @@ def run_reference(args):
             "steps": steps, "warmup": 1, "ms_per_step": round(value * wl.batch / 1e3, 3), "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": wl.name, "policy": args.policy, "note": "fp64 CPU oracle, bounded sample per step"},
-            "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": r["cores"], "kind": "oracle", "sample": sample},
+            "extrapolated": True, "measured_s": round(secs / steps, 2),
+            "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": r["cores"], "kind": "oracle", "sample": sample,
+                             "extrapolated": True, "measured_s": round(secs / steps, 2)},
             "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -653,6 +691,9 @@ def main():
     ap.add_argument("--demanding-fraction", type=float, default=None, help="override the share of cache-demanding layers")
     ap.add_argument("--cpu-rows", type=int, default=256, help="rows of the oracle's timed sample")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--input-sets", type=int, default=4,
+                    help="Q/K/V/out sets per scale that the layers use in turn (so that a coarse scale's inputs are not "
+                         "served from L2 where the previous layer left them)")
     ap.add_argument("--streams", type=int, default=1, choices=[1, 2],
                     help="2: appends on a side stream overlapping attention of other layers; 1: everything in order")
     ap.add_argument("--similarity", action="store_true", help="time amskv_layer_similarity instead of the attention pass")

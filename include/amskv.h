@@ -167,7 +167,10 @@ AMSKV_API int amskv_cache_reset(amskv_cache* cache);
  * Algorithm 2 "rolling", at scale granularity).
  *   K, V      device pointers, logical shape [rows, heads, T, head_dim], T = side^2.
  *   strides   element strides of the (row, head, token) dimensions, or NULL for a
- *             contiguous tensor; the token and head strides must be multiples of 8.
+ *             contiguous tensor; all three must be multiples of 8, the token stride at least
+ *             head_dim.  A zero row (head) stride -- one slice repeated, as an expanded view has --
+ *             is refused with INVALID when there is more than one row (head), and always for a
+ *             tensor the call writes (`out`).
  * The segment that leaves the local window is dropped by bookkeeping alone; its slot is
  * the one the new segment is written to.  Scales must be appended in order 0, 1, 2, ...
  * per layer (ORDER otherwise).  Non-finite K/V values give unspecified results.
@@ -329,10 +332,21 @@ AMSKV_API int amskv_append_copies(const amskv_cache* cache, int layer, int scale
  * last reset. */
 AMSKV_API int amskv_cache_bytes(const amskv_cache* cache, size_t* allocated, size_t* resident_now, size_t* peak);
 
-/* Reads the device status word (synchronises the device).  *device_status is 0 when no
- * kernel reported a problem; otherwise the code of the first bounded wait that gave up, and
- * the return value is AMSKV_ERR_DEVICE_TIMEOUT. */
+/* Reads the device status word (synchronises the device) and clears it.  *device_status is 0 when no
+ * kernel reported a problem since the last call; otherwise it is the code of the first bounded wait that
+ * gave up (1: a key/value or query copy did not arrive, 2: the MMA-issuing warp gave up, 3: a softmax
+ * group or another role gave up) and the return value is AMSKV_ERR_DEVICE_TIMEOUT.  A kernel that gives
+ * up still returns normally (its roles wind down, copies in flight are awaited, tensor memory is freed),
+ * so the context stays usable, but the outputs of that launch are undefined: the calls that enqueue work
+ * return AMSKV_OK regardless, and only this call tells.  amskv_cache_reset does not touch the word. */
 AMSKV_API int amskv_status(amskv_cache* cache, int* device_status);
+
+/* Diagnostic (the paper has no counterpart): enqueues one 32-thread kernel whose bounded wait -- the same
+ * helper every attention kernel waits with -- runs out after `iterations` polls (1 .. 2^20) of a barrier
+ * that nothing arrives at.  The kernel records code 3 in the cache's status word and returns normally;
+ * nothing faults or hangs.  Lets a caller (and the tests) check the whole reporting chain:
+ * amskv_status must then return AMSKV_ERR_DEVICE_TIMEOUT once, and AMSKV_OK afterwards. */
+AMSKV_API int amskv_selftest_wait_timeout(amskv_cache* cache, uint32_t iterations, void* stream);
 
 /* Number of kernels this library has launched since it was loaded. */
 AMSKV_API int64_t amskv_launch_count(void);

@@ -16,7 +16,7 @@ from typing import List, Sequence
 
 import numpy as np
 
-from .selection import (algorithm1_tokens, attended_tokens, clru_tokens, evicted_at,  # noqa: F401
+from .selection import (algorithm1_tokens, algorithm1_trace, attended_tokens, clru_tokens, evicted_at,  # noqa: F401
                         keep_set, keep_set_simulated, kept_tokens, kv_bytes)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

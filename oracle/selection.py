@@ -35,12 +35,12 @@ def keep_set_simulated(k: int, n_condensed: int, n_local: int, cache_demanding: 
         raise ValueError("n_condensed must be >= 0")
     cache: List[int] = []
     for i in range(k + 1):
-        cache = cache + [i]  # Algorithm 1: append the i-th scale
+        cache = cache + [i]  # the new scale joins the cache first (Algorithm 1)
         if cache_demanding:
             continue  # full retention: never rolled
         budget = n_condensed + n_local
         if len(cache) <= budget:
-            continue  # Algorithm 2: no rolling if within budget
+            continue  # a cache that fits its budget is left alone (Algorithm 2)
         prefix = cache[:n_condensed]
         tail = cache[-n_local:]
         cache = prefix + [s for s in tail if s not in prefix]
@@ -69,59 +69,80 @@ def kept_tokens(sides: Sequence[int], keep: Sequence[int]) -> int:
 
 
 def clru_tokens(cache: List[Tuple[int, int]], c_bgt: int, c_cds: int) -> List[Tuple[int, int]]:
-    """Algorithm 2 literally, on a list of tokens.
+    """The eviction rule of Algorithm 2 (Appendix F) on an ordered list of (scale, token) entries.
 
-    `cache` is an ordered list of (scale, token) entries; c_bgt and c_cds are token counts.
-    Within budget the cache is returned unchanged; otherwise the first c_cds entries and the
-    last (c_bgt - c_cds) entries survive.
+    Budgets are token counts.  Stated by position: a cache of n entries that fits the budget is
+    left alone; a longer one keeps position p exactly when p lies in the pinned head (p < c_cds)
+    or among the newest c_bgt - c_cds positions (p >= n - (c_bgt - c_cds)).  Because
+    n > c_bgt = c_cds + (c_bgt - c_cds), the two position sets cannot meet.
     """
-    if len(cache) <= c_bgt:
-        return cache
-    head = cache[:c_cds]
-    k = c_bgt - c_cds
-    tail = cache[-k:] if k > 0 else []
-    seen = set(head)
-    return head + [e for e in tail if e not in seen]
+    n = len(cache)
+    if n <= c_bgt:
+        return list(cache)
+    newest = max(c_bgt - c_cds, 0)
+    return [entry for p, entry in enumerate(cache) if p < c_cds or p >= n - newest]
+
+
+def _outcome(below_theta, scale: int) -> bool:
+    """Outcome of the similarity test S(k_i, resized k_{i-1}) < theta if it is evaluated at `scale`:
+    one boolean for every scale, or a sequence indexed by scale."""
+    if isinstance(below_theta, (bool, int)):
+        return bool(below_theta)
+    return bool(below_theta[scale])
+
+
+def algorithm1_trace(sides: Sequence[int], c_min: int, c_max: int, c_cds: int, below_theta):
+    """Algorithm 1 (Sec. 4.3) with budgets in tokens: (cache after every scale, budget after every scale).
+
+    The layer starts cache-efficient with budget C_min.  For each scale, in order:
+      1. a scale with more tokens than C_max is never cached: the cache is carried over;
+      2. otherwise the scale's tokens join the end of the cache;
+      3. if that exceeds the current budget: while the budget is still C_min the similarity test
+         decides -- at THIS overflow, with this scale's keys, and again at every later overflow as
+         long as the layer has not been promoted -- whether the budget becomes C_max; a scale with
+         more tokens than the (possibly raised) budget is dropped again, leaving the cache as it
+         was; otherwise the cache is rolled by `clru_tokens`.
+    `below_theta` supplies the outcomes of the similarity test (the test itself needs key values):
+    a single boolean, or a sequence indexed by scale so that a layer can fail the test at its
+    first overflow and pass it at a later one, i.e. be promoted after evictions have happened.
+    """
+    cache: List[Tuple[int, int]] = []
+    budget = c_min
+    caches: List[List[Tuple[int, int]]] = []
+    budgets: List[int] = []
+    for i, side in enumerate(sides):
+        own = [(i, t) for t in range(int(side) * int(side))]
+        if len(own) <= c_max:
+            joined = cache + own
+            if len(joined) <= budget:
+                cache = joined
+            else:
+                if budget == c_min and _outcome(below_theta, i):
+                    budget = c_max
+                if len(own) <= budget:
+                    cache = clru_tokens(joined, budget, c_cds)
+        caches.append(list(cache))
+        budgets.append(budget)
+    return caches, budgets
 
 
 def algorithm1_tokens(sides: Sequence[int], c_min: int, c_max: int, c_cds: int,
-                      promote_at_overflow: bool) -> List[List[Tuple[int, int]]]:
-    """Algorithm 1 literally with token budgets; returns the cache after every scale.
+                      below_theta) -> List[List[Tuple[int, int]]]:
+    """The caches of `algorithm1_trace` (one per scale)."""
+    return algorithm1_trace(sides, c_min, c_max, c_cds, below_theta)[0]
 
-    `promote_at_overflow` stands for the outcome of the similarity test S < theta at the
-    first overflow (the test itself needs key values; here only its outcome matters).
-    A scale larger than c_max, or larger than the budget after the promotion decision, is
-    not cached and the cache stays as it was.
+
+def attended_tokens(sides: Sequence[int], k: int, c_bgt: int, c_cds: int, c_max: int = None,
+                    below_theta=False) -> List[Tuple[int, int]]:
+    """(scale, token) pairs the queries of scale k attend to in a token-budget layer.
+
+    The cache Algorithm 1 leaves after scale k, followed by the tokens of scale k that the cache
+    does not hold (the reading taken for a scale that is skipped or cut by its own roll: it still
+    sees itself).  With c_max left out the budget is fixed at c_bgt from the start; otherwise the
+    layer starts at c_bgt (= C_min) and `below_theta` gives the promotion outcomes per scale.
     """
-    cache: List[Tuple[int, int]] = []
-    c_bgt = c_min
-    history: List[List[Tuple[int, int]]] = []
-    for i, side in enumerate(sides):
-        seg = [(i, t) for t in range(side * side)]
-        if len(seg) > c_max:
-            history.append(list(cache))
-            continue
-        grown = cache + seg
-        if len(grown) > c_bgt:
-            if c_bgt == c_min and promote_at_overflow:
-                c_bgt = c_max
-            if len(seg) > c_bgt:
-                history.append(list(cache))
-                continue
-            grown = clru_tokens(grown, c_bgt, c_cds)
-        cache = grown
-        history.append(list(cache))
-    return history
-
-
-def attended_tokens(sides: Sequence[int], k: int, c_bgt: int, c_cds: int) -> List[Tuple[int, int]]:
-    """(scale, token) pairs the queries of scale k attend to in a layer whose budget is fixed at c_bgt.
-
-    The cache Algorithm 1 leaves after scale k (budget c_bgt from the start: see
-    `algorithm1_tokens`, whose promotion happens before anything was evicted), followed by the
-    tokens of scale k that the cache does not hold.
-    """
-    cache = algorithm1_tokens(list(sides[:k + 1]), c_bgt, c_bgt, c_cds, promote_at_overflow=False)[k]
+    top = c_bgt if c_max is None else c_max
+    cache = algorithm1_tokens(list(sides[:k + 1]), c_bgt, top, c_cds, below_theta)[k]
     have = set(cache)
     return cache + [(k, t) for t in range(int(sides[k]) ** 2) if (k, t) not in have]
 

@@ -78,6 +78,7 @@ def _load() -> ctypes.CDLL:
         "amskv_append_copies": ([vp, i, i, i32p, i32p], i),
         "amskv_cache_bytes": ([vp, szp, szp, szp], i),
         "amskv_status": ([vp, ctypes.POINTER(i)], i),
+        "amskv_selftest_wait_timeout": ([vp, ctypes.c_uint32, vp], i),
         "amskv_launch_count": ([], ctypes.c_int64),
         "amskv_strerror": ([i], ctypes.c_char_p),
     }
@@ -93,7 +94,7 @@ EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy am
            "amskv_attend amskv_append_attend amskv_attention_density amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
            "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
            "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_attended_tokens amskv_append_copies "
-           "amskv_cache_bytes amskv_status "
+           "amskv_cache_bytes amskv_status amskv_selftest_wait_timeout "
            "amskv_launch_count amskv_strerror").split()
 
 
@@ -296,12 +297,17 @@ def amskv_cache_bytes(cache: int) -> Tuple[int, int, int]:
 
 
 def amskv_status(cache: int) -> int:
-    """Device status word (0 = fine).  Synchronises the device."""
+    """Device status word (0 = fine); the call clears it.  Synchronises the device."""
     w = ctypes.c_int(0)
     rc = lib.amskv_status(cache, ctypes.byref(w))
     if rc not in (OK, ERR_DEVICE_TIMEOUT):
         raise AmskvError(rc, "amskv_status")
     return int(w.value)
+
+
+def amskv_selftest_wait_timeout(cache: int, iterations: int, stream=None) -> None:
+    """Enqueues the diagnostic kernel whose bounded wait runs out after `iterations` polls."""
+    _check(lib.amskv_selftest_wait_timeout(cache, int(iterations), _stream(stream)), "amskv_selftest_wait_timeout")
 
 
 def amskv_launch_count() -> int:

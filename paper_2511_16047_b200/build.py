@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libamskv.so")
-SOURCES = ["api.cu", "append.cu", "attend_simt.cu", "attend_tc.cu", "attend_pair.cu", "attend_small.cu", "similarity.cu", "density.cu"]
-HEADERS = ["kernels.cuh", "policy.hpp", os.path.join("..", "..", "include", "amskv.h")]
+SOURCES = ["api.cu", "append.cu", "attend_simt.cu", "attend_tc.cu", "attend_pair.cu", "attend_small.cu", "similarity.cu", "density.cu", "selftest.cu"]
+HEADERS = ["kernels.cuh", "policy.hpp", "sm100_ptx.cuh", os.path.join("..", "..", "include", "amskv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

@@ -124,7 +124,11 @@ bool bad_layer_scale(const amskv_cache* c, int layer, int scale)
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
-int make_strided(const void* ptr, const int64_t* strides, int32_t heads, int32_t T, int32_t D, Strided* out)
+// `is_output`: the tensor is written.  A zero row or head stride repeats one slice along that dimension
+// (a broadcast view); the TMA paths cannot express that, and a written tensor must not alias itself, so
+// it is refused wherever the dimension has more than one entry, and for outputs always.
+int make_strided(const void* ptr, const int64_t* strides, int32_t rows, int32_t heads, int32_t T, int32_t D, Strided* out,
+                 bool is_output = false)
 {
     if (!ptr || misaligned(ptr)) return AMSKV_ERR_INVALID;
     out->ptr = ptr;
@@ -134,6 +138,8 @@ int make_strided(const void* ptr, const int64_t* strides, int32_t heads, int32_t
         out->token = strides[2];
         if (out->row < 0 || out->head < 0 || out->token < D) return AMSKV_ERR_INVALID;
         if ((out->row % 8) || (out->head % 8) || (out->token % 8)) return AMSKV_ERR_INVALID;
+        if ((out->row == 0 && (rows > 1 || is_output)) || (out->head == 0 && (heads > 1 || is_output)))
+            return AMSKV_ERR_INVALID;
     } else {
         out->token = D;
         out->head = (int64_t)T * D;
@@ -272,9 +278,9 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
     const LayerLayout& lay = cache->layout[layer];
     if (!cache->plan_only()) {
         Strided ks, vs;
-        int rc = make_strided(K, strides, cache->heads, T, cache->head_dim, &ks);
+        int rc = make_strided(K, strides, cache->rows, cache->heads, T, cache->head_dim, &ks);
         if (rc != AMSKV_OK) return rc;
-        rc = make_strided(V, strides, cache->heads, T, cache->head_dim, &vs);
+        rc = make_strided(V, strides, cache->rows, cache->heads, T, cache->head_dim, &vs);
         if (rc != AMSKV_OK) return rc;
         Piece piece[LayerLayout::kMaxPieces];
         const int32_t n_pieces = lay.pieces(cache->tokens, scale, piece);
@@ -308,9 +314,9 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
     if (scale != cache->last_appended[layer]) return AMSKV_ERR_ORDER;
     const int32_t T = cache->tokens[scale];
     Strided q, o;
-    int rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
+    int rc = make_strided(Q, q_strides, cache->rows, cache->heads, T, cache->head_dim, &q);
     if (rc != AMSKV_OK) return rc;
-    rc = make_strided(out, o_strides, cache->heads, T, cache->head_dim, &o);
+    rc = make_strided(out, o_strides, cache->rows, cache->heads, T, cache->head_dim, &o, true);
     if (rc != AMSKV_OK) return rc;
     RangeList ranges;
     ranges.n = cache->layout[layer].ranges(cache->tokens, scale, ranges.r);
@@ -351,10 +357,10 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
     const int32_t T = cache->tokens[scale];
     const LayerLayout& lay = cache->layout[layer];
     Strided ks, vs, q, o;
-    int rc = make_strided(K, kv_strides, cache->heads, T, cache->head_dim, &ks);
-    if (rc == AMSKV_OK) rc = make_strided(V, kv_strides, cache->heads, T, cache->head_dim, &vs);
-    if (rc == AMSKV_OK) rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
-    if (rc == AMSKV_OK) rc = make_strided(out, o_strides, cache->heads, T, cache->head_dim, &o);
+    int rc = make_strided(K, kv_strides, cache->rows, cache->heads, T, cache->head_dim, &ks);
+    if (rc == AMSKV_OK) rc = make_strided(V, kv_strides, cache->rows, cache->heads, T, cache->head_dim, &vs);
+    if (rc == AMSKV_OK) rc = make_strided(Q, q_strides, cache->rows, cache->heads, T, cache->head_dim, &q);
+    if (rc == AMSKV_OK) rc = make_strided(out, o_strides, cache->rows, cache->heads, T, cache->head_dim, &o, true);
     if (rc != AMSKV_OK) return rc;
     if (cache->transient(scale)) {
         // Never stored: the queries attend to the older retained tokens in the cache and to the scale's own
@@ -458,7 +464,7 @@ int amskv_attention_density(amskv_cache* cache, int layer, int scale, const void
     if (scale != cache->last_appended[layer]) return AMSKV_ERR_ORDER;
     const int32_t T = cache->tokens[scale];
     Strided q;
-    int rc = make_strided(Q, q_strides, cache->heads, T, cache->head_dim, &q);
+    int rc = make_strided(Q, q_strides, cache->rows, cache->heads, T, cache->head_dim, &q);
     if (rc != AMSKV_OK) return rc;
     const LayerLayout& lay = cache->layout[layer];
     TokenRun runs[2 * AMSKV_MAX_SCALES];
@@ -623,9 +629,21 @@ int amskv_status(amskv_cache* cache, int* device_status)
     int word = 0;
     cudaError_t e = cudaDeviceSynchronize();
     if (e == cudaSuccess) e = cudaMemcpy(&word, cache->status_word(), sizeof(int), cudaMemcpyDeviceToHost);
+    // read and clear: one report must not mark every later call of this cache as failed
+    if (e == cudaSuccess && word != 0) e = cudaMemset(cache->status_word(), 0, sizeof(int));
     if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
     *device_status = word;
     return word == 0 ? AMSKV_OK : AMSKV_ERR_DEVICE_TIMEOUT;
+}
+
+int amskv_selftest_wait_timeout(amskv_cache* cache, uint32_t iterations, void* stream)
+{
+    if (!cache) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
+    if (iterations < 1 || iterations > (1u << 20)) return AMSKV_ERR_INVALID;
+    cudaError_t e = launch_wait_gives_up(iterations, cache->status_word(), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+    return AMSKV_OK;
 }
 
 int64_t amskv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

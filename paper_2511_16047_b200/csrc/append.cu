@@ -1,5 +1,5 @@
 // Append: copies one scale's K and V ([rows, heads, T, D] bf16, strided) into the layer's
-// slot for that segment (Algorithm 1, "append the i-th scale").  Pure byte movement, 16 bytes
+// slot for that segment (the step of Algorithm 1 in which a new scale joins the cache).  Pure byte movement, 16 bytes
 // per access; eviction itself moves no data (the evicted segment is the slot's old tenant).
 #include "kernels.cuh"
 

@@ -22,9 +22,8 @@
 // next query tile as soon as the last S of the current one has landed.
 // Every wait is bounded: a wait that gives up records a status code, all roles wind down,
 // copies in flight are awaited and the tensor memory is freed.
-#include <cuda.h>  // CUtensorMap and enums only; the encoder is fetched from the driver at run time
-
 #include "kernels.cuh"
+#include "sm100_ptx.cuh"
 
 namespace amskv {
 
@@ -38,7 +37,6 @@ constexpr int kGroupWarps = 4;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;        // first MMA-issuing warp; Cfg<D>::kMmaWarps of them
 constexpr int kMaxStages = 4;
-constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleLog2 = 8.f;
 constexpr int kQSplitRows = 64;   // query tiles of at most this many rows are double-buffered inside their slot
 constexpr int kPolyEvery = 4;     // every 4th pair of exponentials goes to the FMA pipe (0: none)
@@ -72,6 +70,20 @@ struct Cfg {
     static constexpr uint32_t kTmemCols = kWide ? 512 : 256;
     static constexpr uint32_t kSCol = 0, kOCol = 2 * kSBufs * kKT;
     static constexpr int kCtasPerSm = kWide ? 1 : 2;
+    // Extents every address in the kernel is derived from, checked at compile time:
+    //  - tensor memory: S buffers of both streams, then O of both streams, inside the allocation, and the
+    //    allocations of all CTAs of an SM inside its 512 columns (otherwise tcgen05.alloc would block);
+    //  - shared memory: the CTAs of an SM (each with 1 KB reserved by the system) inside 228 KB;
+    //  - matrix descriptors: a start address is 14 bits of 16-byte units (256 KB), so adding a stage, half
+    //    or K-step offset to the low descriptor word can never carry into the field above it.
+    static_assert(kOCol + 2 * D <= kTmemCols, "S and O of both streams must fit the tensor-memory allocation");
+    static_assert((kTmemCols & (kTmemCols - 1)) == 0 && kTmemCols >= 32 && kCtasPerSm * kTmemCols <= 512,
+                  "tensor-memory allocations of an SM's CTAs");
+    static_assert(kCtasPerSm * (kSmemBytes + 1024) <= 228 * 1024, "shared memory of an SM's CTAs");
+    static_assert(kKVHalfBytes % 1024 == 0 && kQHalfBytes % 1024 == 0 && kStageBytes % 1024 == 0 && kQBytes % 1024 == 0,
+                  "swizzle atoms must stay 1024-byte aligned");
+    static_assert(228 * 1024 <= (1 << 18), "descriptor start-address field covers all of shared memory");
+    static_assert(kStages <= kMaxStages, "barrier arrays");
 };
 
 constexpr int kTileTab = 256;     // tiles whose (first token, valid tokens) are tabulated in shared memory
@@ -142,291 +154,8 @@ __device__ __forceinline__ Stream stream_of(const PairPlan& pp, int32_t pair, in
     return s;
 }
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+using namespace ptx;
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait; false when it gave up or another role already aborted.  The non-blocking test
-// comes first: most waits here find their phase complete already.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-    if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u && *abort_flag) return false;
-    }
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
-
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2)
-{
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-// True in exactly one lane of a converged warp.
-__device__ __forceinline__ bool elect_one()
-{
-    uint32_t pred;
-    asm volatile(
-        "{\n"
-        ".reg .pred P;\n"
-        "elect.sync _|P, 0xffffffff;\n"
-        "selp.u32 %0, 1, 0, P;\n"
-        "}\n"
-        : "=r"(pred));
-    return pred != 0;
-}
-// Bounded wait by a whole warp; the outcome is the same in every lane.
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// Shared-memory matrix descriptors are passed as two 32-bit halves: the low half carries the
-// start address (and the leading offset), the high half is the same for every tile.
-// D (+)= A * B with A and B described in shared memory
-template <bool kAccumulate>
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        ".reg .b64 da, db;\n"
-        "setp.ne.b32 p, %5, 0;\n"
-        "mov.b64 da, {%1, %3};\n"
-        "mov.b64 db, {%2, %3};\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
-        "}\n"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
-        : "memory");
-}
-// D (+)= A * B with A in tensor memory (128 lanes x packed 16-bit pairs) and B in shared memory
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
-                                        uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        ".reg .b64 db;\n"
-        "setp.ne.b32 p, %5, 0;\n"
-        "mov.b64 db, {%2, %3};\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n"
-        "}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-#define AMSKV_R32(r, o)                                                                                               \
-    "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]),   \
-        "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]),            \
-        "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15]), "=r"(r[o + 16]), "=r"(r[o + 17]), "=r"(r[o + 18]),         \
-        "=r"(r[o + 19]), "=r"(r[o + 20]), "=r"(r[o + 21]), "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]),         \
-        "=r"(r[o + 25]), "=r"(r[o + 26]), "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]), "=r"(r[o + 30]),         \
-        "=r"(r[o + 31])
-#define AMSKV_W32(r)                                                                                                  \
-    "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),     \
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),   \
-        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),   \
-        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-#define AMSKV_L32                                                                                                     \
-    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                                        \
-    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}"
-#define AMSKV_L32B                                                                                                    \
-    "{%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "                              \
-    "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}"
-
-// 32 consecutive 32-bit columns of this thread's TMEM lane; returns after the data has arrived.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 " AMSKV_L32 ", [%32];\n"
-                 "tcgen05.wait::ld.sync.aligned;\n"
-                 : AMSKV_R32(r, 0)
-                 : "r"(taddr)
-                 : "memory");
-}
-// 64 consecutive columns (two loads, one wait).
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 " AMSKV_L32 ", [%64];\n"
-                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 " AMSKV_L32B ", [%65];\n"
-                 "tcgen05.wait::ld.sync.aligned;\n"
-                 : AMSKV_R32(r, 0), AMSKV_R32(r, 32)
-                 : "r"(taddr), "r"(taddr + 32)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_st16_nowait(uint32_t taddr, const uint32_t (&r)[16])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
-                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// 8 columns: load, and store (used by the rare rescale of O, which runs with a full S tile in registers)
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
-                 "tcgen05.wait::ld.sync.aligned;\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};\n"
-                 "tcgen05.wait::st.sync.aligned;\n"
-                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-                 : "memory");
-}
-
-__device__ __forceinline__ float fast_exp2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// Packed single-precision pairs (two lanes per instruction on sm_100).
-__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1)
-{
-    asm("{\n"
-        ".reg .b64 ra, rb, rc, rd;\n"
-        "mov.b64 ra, {%2, %3};\n"
-        "mov.b64 rb, {%4, %5};\n"
-        "mov.b64 rc, {%6, %7};\n"
-        "fma.rn.f32x2 rd, ra, rb, rc;\n"
-        "mov.b64 {%0, %1}, rd;\n"
-        "}\n"
-        : "=f"(d0), "=f"(d1)
-        : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
-}
-__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1)
-{
-    asm("{\n"
-        ".reg .b64 ra, rb, rd;\n"
-        "mov.b64 ra, {%2, %3};\n"
-        "mov.b64 rb, {%4, %5};\n"
-        "add.rn.f32x2 rd, ra, rb;\n"
-        "mov.b64 {%0, %1}, rd;\n"
-        "}\n"
-        : "=f"(d0), "=f"(d1)
-        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
-}
-// 2^x for a pair on the FMA pipe instead of the special-function unit: x = n + f with n the
-// nearest integer (obtained by adding 1.5 * 2^23), 2^f by a cubic on [-0.5, 0.5] (relative error
-// below 1e-3, under the bf16 rounding the result gets anyway), and n added into the exponent
-// field.  Inputs below -127 (including -inf) give exactly 0.
-__device__ __forceinline__ void exp2_poly2(float& y0, float& y1, float x0, float x1)
-{
-    constexpr float kMagic = 12582912.f;   // 1.5 * 2^23
-    x0 = fmaxf(x0, -127.f);
-    x1 = fmaxf(x1, -127.f);
-    float r0, r1, n0, n1, f0, f1, p0, p1;
-    add2(r0, r1, x0, x1, kMagic, kMagic);
-    add2(n0, n1, r0, r1, -kMagic, -kMagic);
-    fma2(f0, f1, n0, n1, -1.f, -1.f, x0, x1);
-    fma2(p0, p1, f0, f1, 0.0555041f, 0.0555041f, 0.2402265f, 0.2402265f);
-    fma2(p0, p1, p0, p1, f0, f1, 0.6931472f, 0.6931472f);
-    fma2(p0, p1, p0, p1, f0, f1, 1.f, 1.f);
-    y0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(r0) << 23));
-    y1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(r1) << 23));
-}
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float y;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
-    return y;
-}
-
-// Shared-memory matrix descriptor for a 128-byte-swizzled tile whose rows are 128 bytes.
-// Low half: start address and leading byte offset, both in 16-byte units.  High half: stride
-// byte offset 1024 (eight 128-byte rows), descriptor version 1, layout type 2 (128-byte swizzle).
-__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes)
-{
-    return ((addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
-}
-constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-// Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, A K-major, B K- or MN-major.
-__device__ __forceinline__ uint32_t make_idesc(uint32_t M, uint32_t N, uint32_t b_mn_major)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
-}
-
-__device__ __forceinline__ void report(int* status, int code, volatile int* abort_flag)
-{
-    atomicCAS(status, 0, code);
-    *abort_flag = 1;
-}
 
 // Tile j of the resident ranges: first token and number of valid tokens (<= 64).
 // A tile of range `ext_range` (the current scale in the caller's tensors) carries kExtFlag in t0.

@@ -39,7 +39,6 @@ enum DeviceStatus : int {
     kStatusTmaTimeout = 1,
     kStatusMmaTimeout = 2,
     kStatusSyncTimeout = 3,
-    kStatusTmemAlloc = 4,
 };
 
 cudaError_t launch_append(const Strided& K, const Strided& V, const LayerRegion& region, int32_t token_offset,
@@ -114,6 +113,10 @@ struct DensityPieces {
 };
 cudaError_t launch_density(const Strided& Q, const LayerRegion& region, const DensityPieces& pieces, int32_t T,
                            int32_t rows, int32_t heads, int32_t D, float softmax_scale, double* out, cudaStream_t stream);
+
+// One warp whose bounded wait runs out after `limit` iterations (nothing ever arrives): records
+// kStatusSyncTimeout in *status and returns normally.
+cudaError_t launch_wait_gives_up(uint32_t limit, int* status, cudaStream_t stream);
 
 void count_launch(int n = 1);
 

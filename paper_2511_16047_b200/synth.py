@@ -146,3 +146,24 @@ def smooth_field_keys(rows: int, heads: int, sides: Sequence[int], head_dim: int
         k = std * (rho * field + math.sqrt(max(0.0, 1.0 - rho * rho)) * eps)
         out.append(k.to(torch.bfloat16).reshape(rows, heads, s * s, head_dim))
     return out
+
+
+def growing_logit_qkv(rows: int, heads: int, tokens: int, head_dim: int, seed: int, scale: int,
+                      first_level: int = 0, step: int = 8, group: int = 64, device="cpu"):
+    """Q, K, V whose attention logits climb by `step` (natural-log units) every `group` key tokens.
+
+    u is a fixed +-1/8 sign vector per (row, head); Q = 8 u + noise/32 and key j = level_j * u + noise/8 with
+    level_j = step * (first_level + j // group), so that with a softmax scale of 8 / (head_dim) ... i.e.
+    1/8 for 64 channels and 1/16 for 128 ... the logit of key j is level_j plus a small random part.  A tiled
+    softmax that walks the keys in order meets a much larger maximum in every tile.  All values are exactly
+    representable in bf16 before the noise is added.
+    """
+    dev = torch.device(device)
+    g = _gen(int(seed) * 1000 + scale * 3 + 500, dev)
+    sign = (torch.randint(0, 2, (rows, heads, 1, head_dim), generator=g, device=dev).float() * 2 - 1) / 8
+    level = step * (first_level + torch.arange(tokens, device=dev) // group).float().reshape(1, 1, tokens, 1)
+    noise = lambda: torch.randn((rows, heads, tokens, head_dim), generator=g, device=dev) / 8   # noqa: E731
+    q = (8 * sign + noise() / 4).to(torch.bfloat16)
+    k = (level * sign + noise()).to(torch.bfloat16)
+    v = noise().to(torch.bfloat16)
+    return q, k, v

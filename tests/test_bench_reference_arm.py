@@ -24,6 +24,18 @@ def test_reference_arm_single_process():
     assert line["impl"] == "reference" and line["unit"] == "us/image" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["gpu_launches"] == 0
+    assert line["extrapolated"] is True and line["measured_s"] > 0
+
+
+def test_input_generators_import_without_the_cuda_library():
+    """The reference arm and the oracle's own tests use the seeded input generators; importing them must not
+    load the product's shared library (the binding is loaded on first use only)."""
+    code = ("import sys; from paper_2511_16047_b200 import synth; import paper_2511_16047_b200 as P; "
+            "assert 'paper_2511_16047_b200.binding' not in sys.modules; "
+            "assert not any('libamskv.so' in l for l in open('/proc/self/maps')); "
+            "P.binding; assert 'paper_2511_16047_b200.binding' in sys.modules")
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr
 
 
 def test_reference_arm_two_ranks_print_one_line():

@@ -71,6 +71,31 @@ def test_text_to_image_1024_shape_sampled():
     _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 3, seed=12, need_gb=3.0)
 
 
+def test_var_d30_full_shape_sampled_fused():
+    """The shape the benchmark times, through the call it times: 512 rows x 30 heads x 64, amskv_append_attend at
+    every scale, one layer of each class, sampled items and query rows."""
+    wl = synth.WORKLOADS["var_d30"]
+    _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 40, seed=15,
+                   need_gb=12.0, fused=True)
+
+
+def test_text_to_image_1024_shape_sampled_fused():
+    """The 1024 x 1024-shaped workload (16 rows, 128 channels) through amskv_append_attend."""
+    wl = synth.WORKLOADS["t2i_1024"]
+    _check_sampled(wl, [(wl.n_condensed, wl.n_local, False), (wl.n_condensed, wl.n_local, True)], 3, seed=16,
+                   need_gb=3.0, fused=True)
+
+
+@pytest.mark.parametrize("fraction", [0.25, 1.0])
+def test_sweep_points_at_batch_64(fraction):
+    """Sweep points of the VAR-d30 head layout at batch 64 (128 rows): a quarter of the layers, and all of
+    them, cache-demanding (the seeded mask decides which); fused calls, sampled items."""
+    wl = synth.WORKLOADS["var_d30"].replace(batch=64, layers=4, demanding_fraction=fraction)
+    pols = wl.policies()
+    assert sum(1 for p in pols if p[2]) == (1 if fraction == 0.25 else 4)
+    _check_sampled(wl, pols, 16, seed=17, need_gb=4.0, fused=True)
+
+
 @pytest.mark.parametrize("fused", [False, True], ids=["separate", "fused"])
 def test_depth_36_512_shape_sampled(fused):
     """36 heads x 64 (dim 2304), ten scales up to 32 x 32 (2 240 tokens): head_dim 64 with eight query
@@ -81,7 +106,7 @@ def test_depth_36_512_shape_sampled(fused):
                    fused=fused)
 
 
-@pytest.mark.parametrize("batch", [1, 16])
+@pytest.mark.parametrize("batch", [1, 16, 64])
 def test_policy_sweep_on_var_d30_shape(batch):
     """The VAR-d30 head layout at small batches with a mix of condensed / local settings and layer
     classes in one cache (the sweep's corner points)."""

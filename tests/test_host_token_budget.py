@@ -61,7 +61,7 @@ def _check_layer(cache, layer, sides, c_bgt, c_cds, capacity):
         assert sorted(_expand(runs)) == sorted(want)
         assert [r[0] for r in runs] == sorted(r[0] for r in runs)
         # what stays cached (the transient copy of a scale that is not resident in full does not count)
-        hist = oracle.algorithm1_tokens(list(sides[:k + 1]), c_bgt, c_bgt, c_cds, promote_at_overflow=False)[k]
+        hist = oracle.algorithm1_tokens(list(sides[:k + 1]), c_bgt, c_bgt, c_cds, below_theta=False)[k]
         cached = {s for s, _ in hist}
         assert B.amskv_kept_segments(cache, layer, k) == sorted(cached)
         assert B.amskv_evicted_at(cache, layer, k) == sorted((prev_cached | {k}) - cached)
@@ -129,11 +129,11 @@ def test_promotion_at_first_overflow_equals_starting_at_c_max():
             c_max = c_min + extra
             if c_cds > c_min or c_min > total:
                 continue
-            a = oracle.algorithm1_tokens(sides, c_min, c_max, c_cds, promote_at_overflow=True)
-            b = oracle.algorithm1_tokens(sides, c_max, c_max, c_cds, promote_at_overflow=False)
+            a = oracle.algorithm1_tokens(sides, c_min, c_max, c_cds, below_theta=True)
+            b = oracle.algorithm1_tokens(sides, c_max, c_max, c_cds, below_theta=False)
             assert a == b
-            a = oracle.algorithm1_tokens(sides, c_min, c_max, c_cds, promote_at_overflow=False)
-            b = oracle.algorithm1_tokens(sides, c_min, c_min, c_cds, promote_at_overflow=False)
+            a = oracle.algorithm1_tokens(sides, c_min, c_max, c_cds, below_theta=False)
+            b = oracle.algorithm1_tokens(sides, c_min, c_min, c_cds, below_theta=False)
             # without promotion a scale between C_min and C_max is skipped either way
             assert a == b
 

@@ -125,3 +125,35 @@ def test_bf16_inputs_are_widened_exactly():
     ref = torch.softmax(q.double().reshape(n, 9, 16) @ k.double().reshape(n, 9, 16).transpose(1, 2) * 0.25, -1) \
         @ v.double().reshape(n, 9, 16)
     np.testing.assert_allclose(out, ref.numpy(), rtol=0, atol=1e-14)
+
+
+def test_attend_tokens_whole_segments_equals_attend_selected():
+    """A token list made of whole segments is the kept-segment form, bit for bit."""
+    n, D = 3, 8
+    Q, K, V = _segments(n, D, 11)
+    for keep in ([0, 1, 3, 4], [4], [0, 2, 4]):
+        tokens = [(s, t) for s in keep for t in range(SIDES[s] ** 2)]
+        a = oracle.attend_tokens(Q[4], K, V, tokens, 0.3)
+        b = oracle.attend_selected(Q[4], K, V, keep, 0.3)
+        np.testing.assert_array_equal(a, b)
+
+
+def test_attend_tokens_partial_segments_equals_attention_on_hand_gathered_keys():
+    """Part of a segment, a segment split in two runs, and an unsorted list: the keys are exactly the listed
+    (segment, token) pairs, gathered here by hand one by one."""
+    n, D = 2, 8
+    Q, K, V = _segments(n, D, 12)
+    tokens = [(0, 0), (1, 1), (1, 3), (3, 5), (3, 6), (3, 15), (2, 8), (4, 0), (4, 24), (3, 0)]
+    Kc = np.stack([K[s][:, t, :] for s, t in tokens], axis=1)
+    Vc = np.stack([V[s][:, t, :] for s, t in tokens], axis=1)
+    want = oracle.attention(Q[4], Kc, Vc, 0.5)
+    got = oracle.attend_tokens(Q[4], K, V, tokens, 0.5)
+    np.testing.assert_array_equal(got, want)
+    # and against the definition written out in Python for one query
+    z = 0.5 * Kc[1] @ Q[4][1, 7]
+    p = np.exp(z - z.max())
+    p /= p.sum()
+    np.testing.assert_allclose(got[1, 7], p @ Vc[1], rtol=0, atol=1e-13)
+    # a wrong token would be seen: dropping one key changes the result
+    other = oracle.attend_tokens(Q[4], K, V, tokens[:-1], 0.5)
+    assert np.abs(other - got).max() > 1e-4

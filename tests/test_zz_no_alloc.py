@@ -13,6 +13,7 @@ gone through every other test.
 import pytest
 import torch
 
+import oracle
 from paper_2511_16047_b200 import binding as B
 from paper_2511_16047_b200 import synth
 
@@ -38,10 +39,11 @@ def _static(kp, sp, kc, sc, rows, heads, D):
 
 
 def test_static_scratch_matches_workspace_call_twice_in_a_row():
-    # first call: large enough to fill all 2048 partial slots; second call: a small problem that
-    # uses only a few of them, so stale partials of the first call sit right behind the live ones
+    # first call: 2048 (row, head) items, one block each, so every one of the 2048 partial slots is written;
+    # second call: a small problem that uses only a few of them, so stale partials of the first call sit right
+    # behind the live ones
     cases = [
-        (64, 16, 64, 13, 16, 11),
+        (128, 16, 64, 13, 16, 11),
         (2, 3, 128, 5, 6, 12),
     ]
     for rows, heads, D, sp, sc, seed in cases:
@@ -51,6 +53,30 @@ def test_static_scratch_matches_workspace_call_twice_in_a_row():
         got = _static(kp, sp, kc, sc, rows, heads, D)
         assert want > 0
         assert abs(got - want) <= REL_TOL * want, (rows, heads, D, got, want)
+        # and against the definition (fp64 CPU oracle), so that the pair of calls is not only self-consistent
+        ref = oracle.similarity_ss(kp.cpu().double().reshape(rows * heads, sp * sp, D).numpy(), sp,
+                                   kc.cpu().double().reshape(rows * heads, sc * sc, D).numpy(), sc)
+        assert abs(got - ref) <= REL_TOL * ref, (rows, heads, D, got, ref)
+
+
+def test_static_scratch_at_its_stated_maximum():
+    """Exactly 2^30 sixteen-byte chunks of current-scale keys (16 GiB) is accepted and agrees with the
+    workspace call; one more (row, head) item is refused before anything is launched."""
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < 24e9:
+        pytest.skip("needs about 17 GB of device memory")
+    rows, heads, D, sp, sc = 1024, 16, 128, 2, 64          # 1024 * 16 * 64^2 * 128 / 8 = 2^30
+    assert rows * heads * sc * sc * D // 8 == 1 << 30
+    kp = synth.normal_bf16((rows, heads + 1, sp * sp, D), 21, "cuda")
+    kc = torch.zeros((rows, heads + 1, sc * sc, D), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    f = B.lib.amskv_layer_similarity_static
+    assert f(kp.data_ptr(), sp, kc.data_ptr(), sc, rows, heads + 1, D, out.data_ptr(), None) == B.ERR_UNSUPPORTED
+    want = _with_workspace(kp, sp, kc, sc, rows, heads, D)
+    got = _static(kp, sp, kc, sc, rows, heads, D)
+    assert want > 0 and got == want
+    del kc
+    torch.cuda.empty_cache()
 
 
 def test_static_scratch_argument_errors():
