@@ -13,7 +13,8 @@ import os
 from typing import List, Optional, Sequence, Tuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libamskv.so")
+# AMSKV_LIBRARY names another build of the same library (a debug build, say); default: the in-tree one
+LIB_PATH = os.environ.get("AMSKV_LIBRARY") or os.path.join(_HERE, "libamskv.so")
 
 OK = 0
 ERR_INVALID, ERR_ORDER, ERR_NOMEM, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = -1, -2, -3, -4, -5, -6
