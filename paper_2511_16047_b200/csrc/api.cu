@@ -394,8 +394,26 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
     for (int i = 0; i < after.n; ++i) after.total += after.r[i].len;
     Piece piece[LayerLayout::kMaxPieces];
     const int32_t n_pieces = lay.pieces(cache->tokens, scale, piece);
-    bool fused = cache->tc_ready && choose_kernel(cache, T, after.total) == AttendKernel::Pair && n_pieces == 1 &&
-                 piece[0].src == 0 && piece[0].len == T;
+    const bool one_copy = n_pieces == 1 && piece[0].src == 0 && piece[0].len == T;
+    AttendKernel kernel = choose_kernel(cache, T, after.total);
+    // a single-token scale that is its own only key (the first scale): out = V, one copy kernel does both calls
+    if (cache->path == AMSKV_PATH_AUTO && T == 1 && after.total == 1) kernel = AttendKernel::Small;
+    if (kernel == AttendKernel::Small && one_copy) {
+        // the warp-per-item kernel reads the scale from K and V and stores it on the way
+        RangeList before;
+        before.n = lay.ranges_before(cache->tokens, scale, before.r);
+        before.total = 0;
+        for (int i = 0; i < before.n; ++i) before.total += before.r[i].len;
+        if (before.total + T == after.total) {
+            CurrentScaleSource cur{ks, vs, true, piece[0].dst, cache->region(layer)};
+            cudaError_t e = launch_attend_small(q, o, cache->region(layer), before, T, cache->rows, cache->heads, cache->head_dim,
+                                                cache->softmax_scale, static_cast<cudaStream_t>(stream), &cur);
+            if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+            note_appended(cache, layer, scale);
+            return AMSKV_OK;
+        }
+    }
+    bool fused = cache->tc_ready && kernel == AttendKernel::Pair && one_copy;
     RangeList ranges;
     if (fused) {
         ranges.n = lay.ranges_before(cache->tokens, scale, ranges.r);

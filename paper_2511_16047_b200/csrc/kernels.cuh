@@ -99,9 +99,12 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
 constexpr int kSmallMaxKeys = 32;
 constexpr int kSmallMaxQueries = 16;
 bool small_supported(int32_t T, int32_t total_keys);
+// With `cur`, `ranges` lists the cached keys only and the current scale's T tokens come from the caller's
+// tensors (and are written to position cur->dst of the region when cur->store is set): T plus the cached
+// keys must fit the limits.  A single-token scale that is its own only key is served by a copy kernel.
 cudaError_t launch_attend_small(const Strided& Q, const Strided& O, const LayerRegion& region, const RangeList& ranges,
                                 int32_t T, int32_t rows, int32_t heads, int32_t D, float softmax_scale,
-                                cudaStream_t stream);
+                                cudaStream_t stream, const CurrentScaleSource* cur = nullptr);
 
 // Attention density: the pieces of the per-item region that hold the attended tokens, each with the run
 // (of the attended-token list) it belongs to and the weight 1 / (tokens of that run).
