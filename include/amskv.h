@@ -97,9 +97,16 @@ typedef struct amskv_cache amskv_cache; /* opaque; owned by the library */
  *                    scales; the ablation in Appendix A uses 0, 1 and 2).
  *   n_local          w >= 1: the w most recent scales are kept, the just-appended one
  *                    included (Algorithm 2 keeps the tail of the cache after the append).
- *   cache_demanding  non-zero: the layer keeps every scale (full retention).
+ *   cache_demanding  AMSKV_LAYER_EFFICIENT (0), AMSKV_LAYER_DEMANDING (1): the layer keeps every scale
+ *                    (full retention), or AMSKV_LAYER_PROMOTABLE (2): the layer starts cache-efficient
+ *                    and amskv_promote_layer may make it cache-demanding until its first eviction
+ *                    (Algorithm 1 decides at the first overflow).  A promotable layer's region is sized
+ *                    and laid out like a cache-demanding layer's, whether or not it is promoted.
  * A cache-efficient layer keeps scale s at step k iff s < c or s > k - w.
  */
+#define AMSKV_LAYER_EFFICIENT 0
+#define AMSKV_LAYER_DEMANDING 1
+#define AMSKV_LAYER_PROMOTABLE 2
 typedef struct {
     int32_t n_condensed;
     int32_t n_local;
@@ -117,6 +124,10 @@ typedef struct {
  *                     its amskv_layer_policy (whole scales) instead.
  *   condensed_tokens  C_cds >= 0 in tokens (clamped to the budget): the first C_cds cached
  *                     tokens are pinned.
+ *   promoted_budget_tokens  0, or C_max >= budget_tokens: the layer starts with budget_tokens (C_min)
+ *                     and amskv_promote_layer may raise its budget to this value until its first
+ *                     overflow, as Algorithm 1 does when S < theta there.  The region is sized for
+ *                     the larger of the two layouts.
  * After the append of a scale the cache holds every cached token while their number is within
  * the budget, else the first C_cds of them and the most recent C_bgt - C_cds: the tail may end
  * inside a scale.  A scale with more tokens than the budget is never cached (Algorithm 1 skips
@@ -127,6 +138,7 @@ typedef struct {
 typedef struct {
     int32_t budget_tokens;
     int32_t condensed_tokens;
+    int32_t promoted_budget_tokens;
 } amskv_token_budget;
 
 typedef struct {
@@ -159,7 +171,7 @@ AMSKV_API int amskv_cache_create(const amskv_desc* desc, void* dev_mem, size_t d
 /* Free the object, and the arena only if the library allocated it. */
 AMSKV_API int amskv_cache_destroy(amskv_cache* cache);
 
-/* Forget all appended scales (start a new batch of images).  Metadata only. */
+/* Forget all appended scales (start a new batch of images) and undo promotions.  Metadata only. */
 AMSKV_API int amskv_cache_reset(amskv_cache* cache);
 
 /*
@@ -229,6 +241,25 @@ AMSKV_API int amskv_append_attend(amskv_cache* cache, int layer, int scale, cons
  */
 AMSKV_API int amskv_attention_density(amskv_cache* cache, int layer, int scale, const void* Q,
                                       const int64_t q_strides[3], double* out, size_t out_entries, void* stream);
+
+/*
+ * On-line promotion (Sec. 4.3, Algorithm 1: when the cache first exceeds the budget C_min and the
+ * similarity S(k_i, resized k_{i-1}) of the arriving scale is below theta, the budget becomes C_max).
+ * amskv_first_overflow_scale reports the scale i whose append is the first to exceed the layer's budget
+ * (n_scales if none does): the caller computes S for that scale with amskv_layer_similarity (it holds
+ * K_i, and K_{i-1} from the previous step), compares it with theta (amskv_classify_by_threshold) and, if
+ * the layer is cache-demanding, calls amskv_promote_layer BEFORE appending scale i.  A layer created
+ * AMSKV_LAYER_PROMOTABLE then keeps every scale; a token-budget layer with promoted_budget_tokens gets
+ * that budget.  Host-only, metadata only: nothing has been evicted yet and every cached token already
+ * sits where the larger layout expects it.
+ * Scope: Algorithm 1 repeats the test at every later overflow while the budget is still C_min; this
+ * library takes the decision at the first overflow only -- after an eviction the call is refused.
+ * Errors: UNSUPPORTED (the layer was not created promotable), ORDER (the overflowing scale has already
+ * been appended); promoting twice is harmless.  amskv_cache_reset returns every layer to the class it
+ * was created with.
+ */
+AMSKV_API int amskv_first_overflow_scale(const amskv_cache* cache, int layer, int* scale);
+AMSKV_API int amskv_promote_layer(amskv_cache* cache, int layer);
 
 /* Choose the kernel used by amskv_attend (AMSKV_PATH_*).  The default is AUTO. */
 AMSKV_API int amskv_set_attend_path(amskv_cache* cache, int path);

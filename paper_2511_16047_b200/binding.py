@@ -23,6 +23,7 @@ FLAG_PLAN_ONLY = 1
 FLAG_BULK_APPEND = 2
 FLAG_TRANSIENT_LAST_SCALE = 4
 PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_PAIR, PATH_SMALL = 0, 1, 2, 3, 4
+LAYER_EFFICIENT, LAYER_DEMANDING, LAYER_PROMOTABLE = 0, 1, 2
 
 
 class LayerPolicy(ctypes.Structure):
@@ -30,7 +31,8 @@ class LayerPolicy(ctypes.Structure):
 
 
 class TokenBudget(ctypes.Structure):
-    _fields_ = [("budget_tokens", ctypes.c_int32), ("condensed_tokens", ctypes.c_int32)]
+    _fields_ = [("budget_tokens", ctypes.c_int32), ("condensed_tokens", ctypes.c_int32),
+                ("promoted_budget_tokens", ctypes.c_int32)]
 
 
 class Desc(ctypes.Structure):
@@ -65,6 +67,8 @@ def _load() -> ctypes.CDLL:
         "amskv_append_attend": ([vp, i, i, vp, vp, i64p, vp, vp, i64p, i64p, vp], i),
         "amskv_attention_density": ([vp, i, i, vp, i64p, vp, sz, vp], i),
         "amskv_set_attend_path": ([vp, i], i),
+        "amskv_first_overflow_scale": ([vp, i, ctypes.POINTER(i)], i),
+        "amskv_promote_layer": ([vp, i], i),
         "amskv_step_host": ([vp, i, i, vp, vp, vp, vp, vp, sz, vp], i),
         "amskv_step_staging_bytes": ([vp, szp], i),
         "amskv_layer_similarity": ([vp, i, vp, i, i, i, i, vp, vp, sz, vp], i),
@@ -92,7 +96,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy amskv_cache_reset amskv_append "
-           "amskv_attend amskv_append_attend amskv_attention_density amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
+           "amskv_attend amskv_append_attend amskv_attention_density amskv_first_overflow_scale amskv_promote_layer amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
            "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
            "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_attended_tokens amskv_append_copies "
            "amskv_cache_bytes amskv_status amskv_selftest_wait_timeout "
@@ -140,14 +144,16 @@ def make_desc(layers: int, heads: int, head_dim: int, rows: int, sides: Sequence
               token_budgets: Optional[Sequence[Tuple[int, int]]] = None):
     """Returns (Desc, keepalive) -- keepalive holds the arrays the descriptor points to.
 
-    token_budgets: optional per-layer (budget_tokens, condensed_tokens); a layer with budget 0
-    follows its entry of `policies`."""
+    token_budgets: optional per-layer (budget_tokens, condensed_tokens[, promoted_budget_tokens]); a layer
+    with budget 0 follows its entry of `policies`."""
     sides_arr = (ctypes.c_int32 * len(sides))(*[int(s) for s in sides])
-    pol_arr = (LayerPolicy * len(policies))(*[LayerPolicy(int(c), int(w), 1 if d else 0) for c, w, d in policies])
+    # the class is False / True, or LAYER_PROMOTABLE
+    pol_arr = (LayerPolicy * len(policies))(*[LayerPolicy(int(c), int(w), int(d)) for c, w, d in policies])
     bud_arr = None
     if token_budgets is not None:
         assert len(token_budgets) == len(policies)
-        bud_arr = (TokenBudget * len(token_budgets))(*[TokenBudget(int(b), int(c)) for b, c in token_budgets])
+        bud_arr = (TokenBudget * len(token_budgets))(*[TokenBudget(int(t[0]), int(t[1]), int(t[2]) if len(t) > 2 else 0)
+                                                       for t in token_budgets])
     d = Desc(layers, heads, head_dim, rows, len(sides), sides_arr, pol_arr, float(softmax_scale), flags,
              bud_arr if bud_arr is not None else ctypes.cast(None, ctypes.POINTER(TokenBudget)))
     return d, (sides_arr, pol_arr, bud_arr)
@@ -168,6 +174,16 @@ def amskv_cache_create(desc: Desc, dev_mem=None, dev_bytes: int = 0) -> int:
 
 def amskv_cache_destroy(cache: int) -> None:
     _check(lib.amskv_cache_destroy(cache), "amskv_cache_destroy")
+
+
+def amskv_first_overflow_scale(cache: int, layer: int) -> int:
+    k = ctypes.c_int(0)
+    _check(lib.amskv_first_overflow_scale(cache, layer, ctypes.byref(k)), "amskv_first_overflow_scale")
+    return int(k.value)
+
+
+def amskv_promote_layer(cache: int, layer: int) -> None:
+    _check(lib.amskv_promote_layer(cache, layer), "amskv_promote_layer")
 
 
 def amskv_cache_reset(cache: int) -> None:

@@ -35,6 +35,8 @@ struct amskv_cache {
     int sm_count = 0;
     std::vector<int32_t> sides, tokens;
     std::vector<LayerLayout> layout;
+    std::vector<LayerLayout> layout0;   // as created: amskv_cache_reset undoes promotions
+    std::vector<uint8_t> promotable, promoted;
     std::vector<size_t> layer_offset;  // bytes from the arena start
     std::vector<int32_t> last_appended;
     std::vector<TensorMapBlob> k_maps, v_maps;      // 16-token boxes
@@ -69,10 +71,13 @@ int check_desc(const amskv_desc* d)
         if (d->scale_sides[i] < 1 || d->scale_sides[i] > 4096) return AMSKV_ERR_INVALID;
     for (int l = 0; l < d->layers; ++l) {
         if (d->token_budget && d->token_budget[l].budget_tokens != 0) {
-            if (d->token_budget[l].budget_tokens < 0 || d->token_budget[l].condensed_tokens < 0) return AMSKV_ERR_INVALID;
+            const amskv_token_budget& b = d->token_budget[l];
+            if (b.budget_tokens < 0 || b.condensed_tokens < 0) return AMSKV_ERR_INVALID;
+            if (b.promoted_budget_tokens != 0 && b.promoted_budget_tokens < b.budget_tokens) return AMSKV_ERR_INVALID;
             continue;  // the layer's scale-granular fields are not used
         }
         if (d->policy[l].n_condensed < 0 || d->policy[l].n_local < 1) return AMSKV_ERR_INVALID;
+        if (d->policy[l].cache_demanding < 0 || d->policy[l].cache_demanding > AMSKV_LAYER_PROMOTABLE) return AMSKV_ERR_INVALID;
     }
     if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND | AMSKV_FLAG_TRANSIENT_LAST_SCALE)) != 0)
         return AMSKV_ERR_INVALID;
@@ -98,21 +103,28 @@ int plan(const amskv_desc* d, amskv_cache* c)
         c->tokens[i] = (int32_t)t;
     }
     c->layout.resize(d->layers);
+    c->promotable.assign(d->layers, 0);
+    c->promoted.assign(d->layers, 0);
     c->layer_offset.resize(d->layers);
     size_t at = kStatusBytes;
     for (int l = 0; l < d->layers; ++l) {
         const bool transient_last = (d->flags & AMSKV_FLAG_TRANSIENT_LAST_SCALE) != 0;
-        if (d->token_budget && d->token_budget[l].budget_tokens > 0)
+        if (d->token_budget && d->token_budget[l].budget_tokens > 0) {
             c->layout[l].build_tokens(c->tokens, d->token_budget[l].budget_tokens, d->token_budget[l].condensed_tokens,
-                                      transient_last);
-        else
+                                      transient_last, d->token_budget[l].promoted_budget_tokens);
+            c->promotable[l] = c->layout[l].c_promoted > 0;
+        } else {
+            const bool may_promote = d->policy[l].cache_demanding == AMSKV_LAYER_PROMOTABLE;
             c->layout[l].build(c->tokens, d->policy[l].n_condensed, d->policy[l].n_local,
-                               d->policy[l].cache_demanding != 0, transient_last);
+                               d->policy[l].cache_demanding == AMSKV_LAYER_DEMANDING, transient_last, may_promote);
+            c->promotable[l] = may_promote && !c->layout[l].full;
+        }
         if ((int64_t)c->layout[l].capacity > (1ll << 30)) return AMSKV_ERR_INVALID;
         c->layer_offset[l] = at;
         at += align_up((size_t)c->layout[l].capacity * c->token_bytes());
     }
     c->arena_bytes = at;
+    c->layout0 = c->layout;
     c->last_appended.assign(d->layers, -1);
     return AMSKV_OK;
 }
@@ -263,6 +275,9 @@ int amskv_cache_reset(amskv_cache* cache)
 {
     if (!cache) return AMSKV_ERR_INVALID;
     std::fill(cache->last_appended.begin(), cache->last_appended.end(), -1);
+    // every layer starts a new batch in the class it was created with (Algorithm 1 starts at C_min)
+    for (int l = 0; l < cache->layers; ++l)
+        if (cache->promoted[l]) { cache->layout[l] = cache->layout0[l]; cache->promoted[l] = 0; }
     cache->resident_now = 0;
     cache->peak = 0;
     return AMSKV_OK;
@@ -295,6 +310,26 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
         }
     }
     note_appended(cache, layer, scale);
+    return AMSKV_OK;
+}
+
+int amskv_first_overflow_scale(const amskv_cache* cache, int layer, int* scale)
+{
+    if (!cache || layer < 0 || layer >= cache->layers || !scale) return AMSKV_ERR_INVALID;
+    *scale = cache->layout[layer].first_overflow(cache->tokens);
+    return AMSKV_OK;
+}
+
+int amskv_promote_layer(amskv_cache* cache, int layer)
+{
+    if (!cache || layer < 0 || layer >= cache->layers) return AMSKV_ERR_INVALID;
+    if (!cache->promotable[layer]) return AMSKV_ERR_UNSUPPORTED;
+    if (cache->promoted[layer]) return AMSKV_OK;
+    // legal until the append that overflows the budget: nothing has been evicted, and every cached token sits
+    // where the larger layout expects it
+    if (cache->last_appended[layer] >= cache->layout[layer].first_overflow(cache->tokens)) return AMSKV_ERR_ORDER;
+    cache->layout[layer].promote(cache->tokens);
+    cache->promoted[layer] = 1;
     return AMSKV_OK;
 }
 

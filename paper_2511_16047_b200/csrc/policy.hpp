@@ -53,13 +53,17 @@ struct LayerLayout {
     // queries read it.
     bool token_mode = false;
     int32_t c_bgt = 0, c_cds = 0;
+    int32_t c_promoted = 0;     // budget the layer may be promoted to (0: none)
     int32_t used = 0;           // positions [0, used) hold cached tokens; the transient slot starts at `used`
     std::vector<uint8_t> cached;      // [n_scales] scale enters the stream (its size fits the budget)
     std::vector<uint8_t> transient;   // [n_scales] scale is read from the transient slot at its own step
     std::vector<int64_t> stream_end;  // [n_scales] stream length after the scale
 
+    // `linear`: the segments sit back to back in scale order whatever the class (the layout of a
+    // cache-demanding layer), so that a cache-efficient layer can be promoted later without moving data: until
+    // then it reads the pinned scales and the window out of that layout and reuses no slot.
     void build(const std::vector<int32_t>& tokens, int32_t n_condensed, int32_t n_local, bool demanding,
-               bool transient_last = false)
+               bool transient_last = false, bool linear = false)
     {
         const int32_t K = (int32_t)tokens.size();
         n_scales = K;
@@ -69,7 +73,7 @@ struct LayerLayout {
         w = std::min(std::max(n_local, 1), K);
         full = demanding || (c + w >= K);
         offset.assign(K, 0);
-        if (full) {
+        if (full || linear) {
             int32_t at = 0;
             for (int32_t s = 0; s < stored; ++s) { offset[s] = at; at += tokens[s]; }
             capacity = skip_last ? std::max(at, kMinCapacity) : at;
@@ -95,7 +99,23 @@ struct LayerLayout {
     // Token-budget form: `budget` = C_bgt (C_max for a cache-demanding layer, C_min otherwise) and
     // `condensed` = C_cds, both in tokens.  Starting a cache-demanding layer at C_max is the same as
     // promoting it at its first overflow, because nothing is evicted before that overflow.
-    void build_tokens(const std::vector<int32_t>& tokens, int32_t budget, int32_t condensed, bool transient_last = false)
+    // `promoted_budget` > budget: the layer may later be given that budget (Algorithm 1's C_max); the region is
+    // sized for whichever of the two layouts needs more.  Before the first overflow both layouts put stream
+    // index g at position g, so switching budgets then moves no data.
+    void build_tokens(const std::vector<int32_t>& tokens, int32_t budget, int32_t condensed, bool transient_last = false,
+                      int32_t promoted_budget = 0)
+    {
+        build_tokens_one(tokens, budget, condensed, transient_last);
+        c_promoted = 0;
+        if (promoted_budget > budget) {
+            LayerLayout alt;
+            alt.build_tokens_one(tokens, promoted_budget, condensed, transient_last);
+            capacity = std::max(capacity, alt.capacity);
+            c_promoted = promoted_budget;
+        }
+    }
+
+    void build_tokens_one(const std::vector<int32_t>& tokens, int32_t budget, int32_t condensed, bool transient_last)
     {
         const int32_t K = (int32_t)tokens.size();
         n_scales = K;
@@ -131,6 +151,34 @@ struct LayerLayout {
         const int64_t stored_stream = skip_last ? (K > 1 ? stream_end[K - 2] : 0) : g;
         used = (int32_t)std::min<int64_t>(stored_stream, c_bgt);
         capacity = skip_last ? std::max(used + slot, kMinCapacity) : used + slot;
+    }
+
+    // Scale whose append is the first to push the cache over its budget (Algorithm 1 takes the promotion
+    // decision there); n_scales if the cache never overflows.
+    int32_t first_overflow(const std::vector<int32_t>& tokens) const
+    {
+        if (!token_mode) return full ? n_scales : std::min(c + w, n_scales);
+        const int32_t top = std::max(c_bgt, c_promoted);
+        int64_t g = 0;
+        for (int32_t s = 0; s < n_scales; ++s) {
+            if (tokens[s] > top) continue;   // never cached under either budget: no overflow test
+            if (g + tokens[s] > c_bgt) return s;
+            g += tokens[s];
+        }
+        return n_scales;
+    }
+
+    // Promotion to the cache-demanding class; legal while nothing has been evicted (the caller checks).
+    void promote(const std::vector<int32_t>& tokens)
+    {
+        if (!token_mode) {
+            full = true;
+            return;
+        }
+        const int32_t cap = capacity;
+        build_tokens_one(tokens, c_promoted, c_cds, skip_last);
+        capacity = std::max(capacity, cap);
+        c_promoted = 0;
     }
 
     int32_t position(int64_t g) const
