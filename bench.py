@@ -666,6 +666,92 @@ def run_similarity(args):
                       "classification": {"lowest_similarity_layers_equal_seeded_independent_layers": chosen == mask}}))
 
 
+def run_density(args):
+    """Attention density as a by-product (amskv_attend_density) against the plain attend pass: the same
+    append + attend steps of the workload, replayed from a CUDA graph, with and without the density output.
+    One JSON line; not the headline metric."""
+    import torch
+    from paper_2511_16047_b200 import binding as B
+    from paper_2511_16047_b200 import synth
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    wl = synth.WORKLOADS[args.workload]
+    if args.batch:
+        wl = wl.replace(batch=args.batch)
+    wl = wl.replace(layers=args.layers or 6)
+    policies = wl.policies(full_retention=args.policy == "full")
+    K, tok = len(wl.sides), wl.tokens
+    qkv = [synth.qkv_for_scale(wl.rows, wl.heads, tok[k], wl.head_dim, wl.seed, k, "cuda") for k in range(K)]
+    outs = [torch.empty_like(q) for q, _, _ in qkv]
+    desc, keep = B.make_desc(wl.layers, wl.heads, wl.head_dim, wl.rows, wl.sides, policies)
+    nbytes = B.amskv_cache_required_bytes(desc)
+    arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    cache = B.amskv_cache_create(desc, arena, nbytes)
+    den = torch.zeros((wl.layers, K, wl.heads, K), dtype=torch.float64, device="cuda")
+
+    def step(with_density, events=None):
+        stream = torch.cuda.current_stream()
+        B.amskv_cache_reset(cache)
+        for k in range(K):
+            q, kk, v = qkv[k]
+            for layer in range(wl.layers):
+                B.amskv_append(cache, layer, k, kk, v, stream)
+                if events is not None:
+                    events[k][layer][0].record(stream)
+                if with_density:
+                    B.amskv_attend_density(cache, layer, k, q, outs[k], den[layer, k], wl.heads * K, stream)
+                else:
+                    B.amskv_attend(cache, layer, k, q, outs[k], stream)
+                if events is not None:
+                    events[k][layer][1].record(stream)
+
+    result = {}
+    for with_density in (False, True):
+        for _ in range(max(args.warmup, 3)):
+            step(with_density)
+        torch.cuda.synchronize()
+        l0 = B.amskv_launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(with_density)
+        launches = B.amskv_launch_count() - l0
+        graph.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream = torch.cuda.current_stream()
+        a.record(stream)
+        for _ in range(args.steps):
+            graph.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        # attention calls alone, per scale: CUDA events around each call in an eager replay
+        events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(wl.layers)]
+                  for _ in range(K)]
+        step(with_density, events)
+        torch.cuda.synchronize()
+        per_scale = [round(sum(e0.elapsed_time(e1) for e0, e1 in events[k]), 4) for k in range(K)]
+        result["with_density" if with_density else "plain"] = {"ms_per_step": round(a.elapsed_time(b) / args.steps, 4),
+                                                               "launches_per_step": launches,
+                                                               "attend_ms_per_scale": per_scale}
+    assert B.amskv_status(cache) == 0
+    # the density of the last scale of layer 0, per retained scale, averaged over heads (what Fig. 5 plots)
+    runs = B.amskv_attended_tokens(cache, 0, K - 1)
+    last = den[0, K - 1].flatten()[:wl.heads * len(runs)].view(wl.heads, len(runs)).mean(dim=0).tolist()
+    B.amskv_cache_destroy(cache)
+    ratio = result["with_density"]["ms_per_step"] / result["plain"]["ms_per_step"]
+    print(json.dumps({"metric": "append + attend pass with the attention density as a by-product vs without", "value": round(ratio, 4),
+                      "unit": "time ratio", "higher_is_better": False, "n_gpus": 1, "steps": args.steps, "dtype": "bf16",
+                      "data": "synthetic",
+                      "config": {"workload": "%s: %d layers, %d rows x %d heads x %d, policy %s" % (
+                          wl.name, wl.layers, wl.rows, wl.heads, wl.head_dim, args.policy)},
+                      "gpu_launches": (result["plain"]["launches_per_step"] + result["with_density"]["launches_per_step"]) * args.steps,
+                      "plain": result["plain"], "with_density": result["with_density"],
+                      "attend_ratio_per_scale": [round(d / p, 3) if p else None for p, d in zip(result["plain"]["attend_ms_per_scale"],
+                                                                                                result["with_density"]["attend_ms_per_scale"])],
+                      "density_of_last_scale_layer_0": {"runs": runs, "mean_over_heads": [round(x, 5) for x in last]}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -697,6 +783,8 @@ def main():
     ap.add_argument("--streams", type=int, default=1, choices=[1, 2],
                     help="2: appends on a side stream overlapping attention of other layers; 1: everything in order")
     ap.add_argument("--similarity", action="store_true", help="time amskv_layer_similarity instead of the attention pass")
+    ap.add_argument("--density", action="store_true",
+                    help="time the append + attend pass with and without the attention density as a by-product")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compare", action="store_true")
@@ -707,6 +795,8 @@ def main():
         run_reference(args)
     elif args.similarity:
         run_similarity(args)
+    elif args.density:
+        run_density(args)
     else:
         run_ours(args)
 

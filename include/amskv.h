@@ -243,6 +243,23 @@ AMSKV_API int amskv_attention_density(amskv_cache* cache, int layer, int scale, 
                                       const int64_t q_strides[3], double* out, size_t out_entries, void* stream);
 
 /*
+ * amskv_attend(layer, scale, Q, out) that also returns the attention density of the same queries (Sec. 4.1,
+ * the definition of d), as a by-product of the attention launch: where the paired tensor-core kernel serves
+ * the scale, its key tiles are cut at the boundaries of the runs of attended tokens, and the un-normalised
+ * probability mass of a query row on a run is a running sum of the per-tile sums the softmax computes anyway;
+ * the rows are normalised by their row sums in the epilogue and added up per (head, run).  One launch, no
+ * second pass over the keys; the cut tiles make the launch somewhat longer than a plain amskv_attend (more,
+ * partly filled key tiles).  `out` is the same as amskv_attend's.  `density`, `density_entries` and the
+ * meaning of the numbers are those of amskv_attention_density (probabilities after their rounding to bf16,
+ * where that call uses them unrounded: they agree to about 1e-4 relative).  Scales the other kernels serve,
+ * and layers with more than 16 runs, run as amskv_attend followed by amskv_attention_density.
+ * Errors: as for the two calls.
+ */
+AMSKV_API int amskv_attend_density(amskv_cache* cache, int layer, int scale, const void* Q, void* out,
+                                   const int64_t q_strides[3], const int64_t o_strides[3], double* density,
+                                   size_t density_entries, void* stream);
+
+/*
  * On-line promotion (Sec. 4.3, Algorithm 1: when the cache first exceeds the budget C_min and the
  * similarity S(k_i, resized k_{i-1}) of the arriving scale is below theta, the budget becomes C_max).
  * amskv_first_overflow_scale reports the scale i whose append is the first to exceed the layer's budget

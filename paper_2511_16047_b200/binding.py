@@ -66,6 +66,7 @@ def _load() -> ctypes.CDLL:
         "amskv_attend": ([vp, i, i, vp, vp, i64p, i64p, vp], i),
         "amskv_append_attend": ([vp, i, i, vp, vp, i64p, vp, vp, i64p, i64p, vp], i),
         "amskv_attention_density": ([vp, i, i, vp, i64p, vp, sz, vp], i),
+        "amskv_attend_density": ([vp, i, i, vp, vp, i64p, i64p, vp, sz, vp], i),
         "amskv_set_attend_path": ([vp, i], i),
         "amskv_first_overflow_scale": ([vp, i, ctypes.POINTER(i)], i),
         "amskv_promote_layer": ([vp, i], i),
@@ -96,7 +97,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("amskv_cache_required_bytes amskv_cache_create amskv_cache_destroy amskv_cache_reset amskv_append "
-           "amskv_attend amskv_append_attend amskv_attention_density amskv_first_overflow_scale amskv_promote_layer amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
+           "amskv_attend amskv_append_attend amskv_attention_density amskv_attend_density amskv_first_overflow_scale amskv_promote_layer amskv_set_attend_path amskv_step_host amskv_step_staging_bytes amskv_layer_similarity "
            "amskv_similarity_workspace_bytes amskv_layer_similarity_static amskv_classify_by_threshold amskv_classify_lowest "
            "amskv_kept_segments amskv_evicted_at amskv_resident_ranges amskv_attended_tokens amskv_append_copies "
            "amskv_cache_bytes amskv_status amskv_selftest_wait_timeout "
@@ -215,6 +216,12 @@ def amskv_attention_density(cache: int, layer: int, scale: int, Q, out, out_entr
     """Attention density per (head, run of amskv_attended_tokens) into `out` (device doubles)."""
     _check(lib.amskv_attention_density(cache, layer, scale, _addr(Q), _strides(Q), _addr(out), int(out_entries),
                                        _stream(stream)), "amskv_attention_density")
+
+
+def amskv_attend_density(cache: int, layer: int, scale: int, Q, out, density, density_entries: int, stream=None) -> None:
+    """amskv_attend plus the attention density of the same queries, from one launch where the paired kernel serves."""
+    _check(lib.amskv_attend_density(cache, layer, scale, _addr(Q), _addr(out), _strides(Q), _strides(out), _addr(density),
+                                    int(density_entries), _stream(stream)), "amskv_attend_density")
 
 
 def amskv_set_attend_path(cache: int, path: int) -> None:

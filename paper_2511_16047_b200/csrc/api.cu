@@ -541,6 +541,55 @@ int amskv_attention_density(amskv_cache* cache, int layer, int scale, const void
     return AMSKV_OK;
 }
 
+int amskv_attend_density(amskv_cache* cache, int layer, int scale, const void* Q, void* out, const int64_t q_strides[3],
+                         const int64_t o_strides[3], double* density, size_t density_entries, void* stream)
+{
+    if (bad_layer_scale(cache, layer, scale) || !density || (reinterpret_cast<uintptr_t>(density) & 7u)) return AMSKV_ERR_INVALID;
+    if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
+    if (scale != cache->last_appended[layer]) return AMSKV_ERR_ORDER;
+    const int32_t T = cache->tokens[scale];
+    Strided q, o;
+    int rc = make_strided(Q, q_strides, cache->rows, cache->heads, T, cache->head_dim, &q);
+    if (rc == AMSKV_OK) rc = make_strided(out, o_strides, cache->rows, cache->heads, T, cache->head_dim, &o, true);
+    if (rc != AMSKV_OK) return rc;
+    const LayerLayout& lay = cache->layout[layer];
+    TokenRun runs[2 * AMSKV_MAX_SCALES];
+    const int32_t n_runs = lay.attended(cache->tokens, scale, runs);
+    if (density_entries < (size_t)cache->heads * (size_t)n_runs) return AMSKV_ERR_NOMEM;
+    LayerLayout::RunPiece rp[kMaxDensityPieces];
+    const int32_t n = lay.attended_pieces(cache->tokens, scale, rp, kMaxDensityPieces);
+    if (n < 0) return AMSKV_ERR_UNSUPPORTED;   // the scale's own keys are not in the cache (never-stored last scale)
+    int32_t total = 0;
+    for (int32_t i = 0; i < n; ++i) total += rp[i].len;
+    // One launch where the paired kernel serves the scale: its key tiles are cut at the boundaries of the runs
+    // (one range per piece of a run), and each row's mass per run falls out of the softmax loop.
+    if (cache->tc_ready && choose_kernel(cache, T, total) == AttendKernel::Pair && n_runs <= kPairMaxDensityRuns && n <= kMaxRanges) {
+        RangeList ranges;
+        PairDensity den;
+        den.out = density;
+        den.n_runs = n_runs;
+        for (int32_t r = 0; r < n_runs; ++r) den.weight[r] = (float)(1.0 / ((double)cache->rows * (double)runs[r].count));
+        ranges.n = n;
+        ranges.total = total;
+        for (int32_t i = 0; i < n; ++i) {
+            ranges.r[i] = Range{rp[i].start, rp[i].len};
+            den.run_of_range[i] = (int8_t)rp[i].run;
+        }
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        cudaError_t e = cudaMemsetAsync(density, 0, sizeof(double) * (size_t)cache->heads * n_runs, st);
+        if (e == cudaSuccess)
+            e = launch_attend_pair(q, o, cache->k_maps[layer].bytes, cache->v_maps[layer].bytes, cache->k_maps64[layer].bytes,
+                                   cache->v_maps64[layer].bytes, ranges, T, cache->rows, cache->heads, cache->head_dim,
+                                   cache->softmax_scale, cache->status_word(), cache->sm_count, st, nullptr, &den);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return AMSKV_ERR_CUDA; }
+        return AMSKV_OK;
+    }
+    // elsewhere (the coarse scales, more runs than the kernel tells apart): the two calls
+    rc = amskv_attend(cache, layer, scale, Q, out, q_strides, o_strides, stream);
+    if (rc != AMSKV_OK) return rc;
+    return amskv_attention_density(cache, layer, scale, Q, q_strides, density, density_entries, stream);
+}
+
 int amskv_step_staging_bytes(const amskv_cache* cache, size_t* bytes)
 {
     if (!cache || !bytes) return AMSKV_ERR_INVALID;

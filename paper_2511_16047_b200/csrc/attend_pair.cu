@@ -30,6 +30,7 @@ namespace amskv {
 namespace {
 
 constexpr int kQRows = 128;       // query rows per tile = TMEM lanes
+constexpr int kMaxDenRuns = 16;   // runs of attended tokens a density launch can tell apart
 constexpr int kQBoxRows = 32;     // query rows per bulk copy
 constexpr int kKT = 64;           // key/value tokens per tile
 constexpr int kKVBoxRows = 16;    // tokens per bulk copy
@@ -44,17 +45,20 @@ constexpr int kPolyEvery = 4;     // every 4th pair of exponentials goes to the 
 // kWide: one CTA per SM with two S buffers per stream and an issuing warp per stream (below): the form
 // 128 channels use.  64 channels use the two-CTA form (the wide form is instantiable for them, but lost
 // wherever it was measured).
-template <int D, bool kWide>
+// kDen: the launch also accumulates the attention density (below): two CTAs per SM then run with three
+// key/value stages, the fourth stage's 16 KB holding the per-row sums.
+template <int D, bool kWide, bool kDen = false>
 struct Cfg {
     static_assert(D == 64 || kWide, "128 channels always use the wide form");
     static constexpr int kHalves = D / 64;                      // 128-byte swizzle atoms per row
-    static constexpr int kStages = 4;
+    static constexpr int kStages = (kDen && !kWide) ? 3 : 4;
     static constexpr uint32_t kQBytes = kQRows * D * 2;         // one query tile
     static constexpr uint32_t kQHalfBytes = kQRows * 128;
     static constexpr uint32_t kKVBytes = kKT * D * 2;           // one K (or V) tile
     static constexpr uint32_t kKVHalfBytes = kKT * 128;
     static constexpr uint32_t kStageBytes = 2 * kKVBytes;
-    static constexpr uint32_t kTileBytes = 2 * kQBytes + kStages * kStageBytes;
+    static constexpr uint32_t kDenBytes = kDen ? 2u * kMaxDenRuns * kQRows * 4u : 0u;   // [stream][run][row] fp32
+    static constexpr uint32_t kTileBytes = 2 * kQBytes + kStages * kStageBytes + kDenBytes;
     static constexpr uint32_t kSmemBytes = 4096 + kTileBytes;   // barriers, tile table and alignment slack in front
     // Score buffers per stream.  With 64 channels two CTAs share the SM's 512 tensor-memory columns and a
     // stream has one S buffer (S and O of two streams: 256 columns).  With 128 channels one CTA has all
@@ -128,6 +132,16 @@ struct ExtArgs {
     int32_t rider_tok, rider_valid;   // older cache tokens that ride in the spare box of the scale's last tile
 };
 
+// Attention density as a by-product (Sec. 4.1): the range list of such a launch has one entry per piece of a
+// run of attended tokens (never merged across runs), so every key tile belongs to one run and a row's
+// un-normalised probability mass per run is a running sum of the tile sums the softmax computes anyway.
+struct DenArgs {
+    double* out;                       // [heads][n_runs], accumulated with atomic adds
+    int32_t n_runs;
+    float weight[kMaxDenRuns];         // 1 / (rows * tokens of the run)
+    int8_t run_of_range[kMaxRanges];
+};
+
 struct Stream {
     int32_t item;
     int32_t qt;
@@ -159,7 +173,8 @@ using namespace ptx;
 
 // Tile j of the resident ranges: first token and number of valid tokens (<= 64).
 // A tile of range `ext_range` (the current scale in the caller's tensors) carries kExtFlag in t0.
-__device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0, int32_t& valid, int ext_range = -1)
+__device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0, int32_t& valid, int ext_range = -1,
+                                        int* range_index = nullptr)
 {
     int r = 0;
     for (; r < rl.n - 1; ++r) {
@@ -170,20 +185,23 @@ __device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0,
     t0 = rl.r[r].start + j * kKT;
     valid = min(kKT, rl.r[r].start + rl.r[r].len - t0);
     if (r == ext_range) t0 |= kExtFlag;
+    if (range_index) *range_index = r;
 }
 
 // ---------------------------------------------------------------- kernel
-template <int D, bool kExt, bool kWide>
-__global__ void __launch_bounds__(Cfg<D, kWide>::kThreads, Cfg<D, kWide>::kCtasPerSm)
+template <int D, bool kExt, bool kWide, bool kDen>
+__global__ void __launch_bounds__(Cfg<D, kWide, kDen>::kThreads, Cfg<D, kWide, kDen>::kCtasPerSm)
 attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap k_map64,
                    const __grid_constant__ CUtensorMap v_map64, const __grid_constant__ ExtArgs ext,
                    __nv_bfloat16* __restrict__ O, int64_t o_row,
                    int64_t o_head, int64_t o_tok, const RangeList ranges, int32_t T, int32_t heads,
-                   const PairPlan pp, int32_t n_tiles, int3 qpos, float scale_log2, int* __restrict__ status)
+                   const PairPlan pp, int32_t n_tiles, int3 qpos, float scale_log2, int* __restrict__ status,
+                   const __grid_constant__ DenArgs den)
 {
+    static_assert(!(kDen && kExt), "the density form serves the plain attend call");
     const int ext_range = kExt ? ext.range : -1;
-    using C = Cfg<D, kWide>;
+    using C = Cfg<D, kWide, kDen>;
     extern __shared__ uint8_t smem_raw[];
     Barriers* bars = reinterpret_cast<Barriers*>(smem_raw);
     volatile int* abort_flag = &bars->abort_flag;
@@ -217,13 +235,18 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
     for (int j = threadIdx.x; j < n_tiles && j < kTileTab; j += C::kThreads) {
         int32_t t0, valid;
-        tile_at(ranges, j, t0, valid, ext_range);
-        bars->tile_tab[j] = make_int2(t0, valid);
+        int ri = 0;
+        tile_at(ranges, j, t0, valid, ext_range, &ri);
+        bars->tile_tab[j] = make_int2(t0, kDen ? (valid | ((int32_t)den.run_of_range[ri] << 8)) : valid);
     }
     if (layout_ok) {
         // query rows a tile does not cover keep whatever the slot held before; start them at zero
         uint4* qz = reinterpret_cast<uint4*>(smem_raw + (q_smem - raw));
         for (uint32_t i = threadIdx.x; i < 2 * C::kQBytes / 16; i += C::kThreads) qz[i] = make_uint4(0, 0, 0, 0);
+        if (kDen) {
+            uint4* dz = reinterpret_cast<uint4*>(smem_raw + (kv_smem - raw) + C::kStages * C::kStageBytes);
+            for (uint32_t i = threadIdx.x; i < C::kDenBytes / 16; i += C::kThreads) dz[i] = make_uint4(0, 0, 0, 0);
+        }
         fence_async_smem();
     }
     if (warp == kProducerWarp) {
@@ -236,14 +259,22 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
+    // (in a density launch `valid` carries the tile's run in its bits 8..15; tile_run() strips it)
     auto tile_of = [&](int j, int32_t& t0, int32_t& valid) {
         if (j < kTileTab) {
             const int2 e = bars->tile_tab[j];
             t0 = e.x;
             valid = e.y;
         } else {
-            tile_at(ranges, j, t0, valid, ext_range);
+            int ri = 0;
+            tile_at(ranges, j, t0, valid, ext_range, &ri);
+            if (kDen) valid |= (int32_t)den.run_of_range[ri] << 8;
         }
+    };
+    auto tile_run = [](int32_t& valid) -> int {
+        const int run = kDen ? (valid >> 8) : 0;
+        if (kDen) valid &= 0xff;
+        return run;
     };
 
     const uint32_t q_full0 = smem_u32(&bars->q_full[0][0]);   // [g][half] at + 16 * g + 8 * half
@@ -305,6 +336,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             for (int j = 0; ok && j < n_tiles; ++j) {
                 int32_t t0, valid;
                 tile_of(j, t0, valid);
+                (void)tile_run(valid);
                 const bool from_ext = kExt && (t0 & kExtFlag) != 0;
                 t0 &= ~kExtFlag;
                 const int nch = (valid + 15) >> 4;
@@ -466,6 +498,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     int32_t t0, valid;
                     tile_of(j, t0, valid);
+                    (void)tile_run(valid);
                     const uint32_t nch = ((uint32_t)(valid + 15) >> 4) +
                                          ((kExt && ext.rider_valid > 0 && j == n_tiles - 1) ? 1u : 0u);
                     const uint32_t idesc_s = make_idesc(kQRows, nch * 16, 0);
@@ -546,6 +579,9 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const uint32_t o_tmem = tmem + C::kOCol + g * D + lane_base;
         const uint32_t o_full = o_full0 + 8 * g;
         const bool q_loader = (wq == 0 && lane == 0);
+        // density: [run][row] sums of this stream, in the shared memory the fourth key/value stage would take
+        // (every thread only ever touches the entries of its own row; they were zeroed before the roles split)
+        float* den_rows = reinterpret_cast<float*>(smem_raw + (kv_smem - raw) + C::kStages * C::kStageBytes) + g * kMaxDenRuns * kQRows;
         uint32_t q_armed = 0;     // query tiles requested so far
         uint32_t q_next_n = 0;    // first pair index not yet searched for a query tile
 
@@ -591,9 +627,18 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             const int32_t valid_rows = min(kQRows, T - st.qt * kQRows);
             const bool warp_live = wq * 32 < valid_rows;
             float m_ref = 0.f, nb = 0.f, l = 0.f;
+            float run_mass = 0.f;   // density: this row's un-normalised mass on the run the tiles are in
+            int cur_run = -1;
             for (int j = 0; j < n_tiles; ++j, ++t) {
                 int32_t t0, valid;
                 tile_of(j, t0, valid);
+                const int run = tile_run(valid);
+                if (kDen && run != cur_run) {
+                    // (the same for every thread: tiles and their runs are launch constants)
+                    if (cur_run >= 0 && warp_live) den_rows[cur_run * kQRows + r] += run_mass;
+                    run_mass = 0.f;
+                    cur_run = run;
+                }
                 const uint32_t s_tmem = s_tmem0 + buf_of(t) * kKT;
                 const uint32_t s_full = s_full0 + 16 * g + 8 * buf_of(t), p_full = p_full0 + 16 * g + 8 * buf_of(t);
                 if (!__all_sync(0xffffffffu, mbar_wait(s_full, par_of(t), abort_flag))) {
@@ -655,6 +700,10 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                                 m_ref = mt;
                                 nb = -mt * scale_log2;
                                 l *= alpha;
+                                if (kDen) {
+                                    run_mass *= alpha;
+                                    for (int rn = 0; rn < den.n_runs; ++rn) den_rows[rn * kQRows + r] *= alpha;
+                                }
                             }
 #pragma unroll 1
                             for (int cblk = 0; cblk < D / 8; ++cblk) {
@@ -690,7 +739,9 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         }
                         tmem_st16_nowait(s_tmem + half * (kKT / 4), pk);
                     }
-                    l += sum0 + sum1;
+                    const float tile_sum = sum0 + sum1;
+                    l += tile_sum;
+                    if (kDen) run_mass += tile_sum;
                     tmem_wait_st();
                 }
                 tc_fence_before();
@@ -727,6 +778,20 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     }
                 }
             }
+            if (kDen && warp_live) {
+                // the row's share of every run, normalised by its row sum, added up over the warp's rows and
+                // then, weighted by 1 / (rows * tokens of the run), into the head's entry of the result
+                if (cur_run >= 0) den_rows[cur_run * kQRows + r] += run_mass;
+                const float inv = (r < valid_rows) ? 1.f / l : 0.f;
+                const int32_t head = st.item % heads;
+                for (int rn = 0; rn < den.n_runs; ++rn) {
+                    float v = den_rows[rn * kQRows + r] * inv;
+                    den_rows[rn * kQRows + r] = 0.f;   // the next unit starts from zero
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                    if (lane == 0) atomicAdd(den.out + (int64_t)head * den.n_runs + rn, (double)v * (double)den.weight[rn]);
+                }
+            }
             tc_fence_before();   // orders the reads of O before the arrival on p_full for the next unit's first tile
             ++un;
         }
@@ -751,21 +816,21 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 }
 
 // ---------------------------------------------------------------- host side
-template <int D, bool kExt, bool kWide>
+template <int D, bool kExt, bool kWide, bool kDen>
 cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& km64,
                    const CUtensorMap& vm64, const ExtArgs& ext, const Strided& O,
                    const RangeList& ranges, int32_t T, int32_t heads, const PairPlan& pp, int32_t n_tiles, int3 qpos,
-                   float scale_log2, int* status, int sm_count, cudaStream_t stream)
+                   float scale_log2, int* status, int sm_count, cudaStream_t stream, const DenArgs& den)
 {
-    using C = Cfg<D, kWide>;
+    using C = Cfg<D, kWide, kDen>;
     static SharedMemoryOptIn opt_in;
-    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide>, (int)C::kSmemBytes);
+    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide, kDen>, (int)C::kSmemBytes);
     if (oe != cudaSuccess) return oe;
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > pp.n_pairs) grid = pp.n_pairs;
-    attend_pair_kernel<D, kExt, kWide><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
+    attend_pair_kernel<D, kExt, kWide, kDen><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
         qm, km, vm, km64, vm64, ext, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos,
-        scale_log2, status);
+        scale_log2, status, den);
     count_launch();
     return cudaGetLastError();
 }
@@ -775,9 +840,22 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
 cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map, const void* v_map,
                                const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
                                float softmax_scale, int* status, int sm_count, cudaStream_t stream,
-                               const CurrentScaleSource* cur)
+                               const CurrentScaleSource* cur, const PairDensity* density)
 {
     if (ranges.n < 1 || ranges.total < 1 || T < 1) return cudaErrorInvalidValue;
+    DenArgs den;
+    memset(&den, 0, sizeof(den));
+    if (density) {
+        static_assert(kPairMaxDensityRuns == kMaxDenRuns, "interface and kernel disagree");
+        if (cur || density->n_runs < 1 || density->n_runs > kMaxDenRuns || !density->out) return cudaErrorInvalidValue;
+        den.out = density->out;
+        den.n_runs = density->n_runs;
+        for (int i = 0; i < density->n_runs; ++i) den.weight[i] = density->weight[i];
+        for (int i = 0; i < ranges.n; ++i) {
+            if (density->run_of_range[i] < 0 || density->run_of_range[i] >= density->n_runs) return cudaErrorInvalidValue;
+            den.run_of_range[i] = density->run_of_range[i];
+        }
+    }
     ExtArgs ext;
     memset(&ext, 0, sizeof(ext));
     ext.range = -1;
@@ -831,15 +909,17 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     // 64 channels always take the two-CTA form: the wide form was measured on the tensor-bound launches of a
     // 2 240-token schedule (T = 576 and 1 024, 36 heads) and lost there too (26.3 vs 20.8 and 64.2 vs 53.9 ms):
     // two streams per SM do not keep the tensor pipe as busy as four, even with the chain broken.
-#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE)                                                                             \
-    return launch<DD, EXT, WIDE>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2, status, \
-                                 sm_count, stream)
+#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE, DEN)                                                                        \
+    return launch<DD, EXT, WIDE, DEN>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2,   \
+                                      status, sm_count, stream, den)
     if (D == 128) {
-        if (cur) AMSKV_PAIR_LAUNCH(128, true, true);
-        AMSKV_PAIR_LAUNCH(128, false, true);
+        if (density) AMSKV_PAIR_LAUNCH(128, false, true, true);
+        if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false);
+        AMSKV_PAIR_LAUNCH(128, false, true, false);
     }
-    if (cur) AMSKV_PAIR_LAUNCH(64, true, false);
-    AMSKV_PAIR_LAUNCH(64, false, false);
+    if (density) AMSKV_PAIR_LAUNCH(64, false, false, true);
+    if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false);
+    AMSKV_PAIR_LAUNCH(64, false, false, false);
 #undef AMSKV_PAIR_LAUNCH
 }
 

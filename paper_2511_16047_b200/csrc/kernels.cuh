@@ -89,11 +89,23 @@ bool tc_encode_q_map(const Strided& Q, int32_t T, int32_t rows, int32_t heads, i
 bool tc_encode_kv_store_maps(const LayerRegion& region, int64_t items, int32_t D, int box_rows, int32_t token_extent,
                              void* k_map_out, void* v_map_out);
 
+// Attention density as a by-product of a paired-kernel launch: `ranges` then has one entry per piece of a run
+// of attended tokens (run_of_range[i] = the run of entry i; entries are never merged across runs), and the
+// launch adds weight[r] * (sum over the item's queries of the normalised probability mass on run r) to
+// out[head * n_runs + r] with atomic adds (out is zeroed by the caller, on the same stream).
+constexpr int kPairMaxDensityRuns = 16;
+struct PairDensity {
+    double* out;
+    int32_t n_runs;
+    float weight[kPairMaxDensityRuns];
+    int8_t run_of_range[kMaxRanges];
+};
+
 // Paired tensor-core kernel: two softmax groups per CTA, probabilities kept in tensor memory.
 cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k_map16, const void* v_map16,
                                const void* k_map64, const void* v_map64, const RangeList& ranges, int32_t T, int32_t rows, int32_t heads, int32_t D,
                                float softmax_scale, int* status, int sm_count, cudaStream_t stream,
-                               const CurrentScaleSource* cur = nullptr);
+                               const CurrentScaleSource* cur = nullptr, const PairDensity* density = nullptr);
 
 // Warp-per-item kernel for the coarse scales: every retained key in one register tile.
 constexpr int kSmallMaxKeys = 32;

@@ -61,3 +61,37 @@ def test_order_and_argument_errors():
         out = torch.zeros(heads * 2, dtype=torch.float64, device="cuda")
         assert B.lib.amskv_attention_density(c.h, 0, 1, q.data_ptr(), None, out.data_ptr(), out.numel(), None) == B.ERR_UNSUPPORTED
         torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("peaked", [False, True], ids=["flat", "peaked"])
+def test_density_as_a_by_product_of_the_attention_launch(D, peaked):
+    """amskv_attend_density: the output equals amskv_attend's bit for bit where both run the paired kernel on
+    the same tiles (and the oracle everywhere), and the density equals the oracle's -- whole scales and token
+    budgets, more units than CTAs, query tiles with idle warps, rows whose reference maximum moves (peaked)."""
+    from gpu_common import check_close, oracle_outputs
+    sides, rows, heads = (1, 2, 3, 5, 6, 8, 13), 6, 40
+    qkv = make_qkv(rows, heads, sides, D, seed=63, peaked=peaked)
+    pols = [(2, 2, False), (2, 2, True), (1, 3, False), (2, 2, False)]
+    budgets = [(0, 0), (0, 0), (0, 0), (120, 5)]
+    scale = 1.0 / math.sqrt(D)
+    Ks = [to_items(k) for _, k, _ in qkv]
+    Vs = [to_items(v) for _, _, v in qkv]
+    with Cache(len(pols), heads, D, rows, sides, pols, token_budgets=budgets) as c:
+        for k, (q, kk, v) in enumerate(qkv):
+            for layer in range(len(pols)):
+                B.amskv_append(c.h, layer, k, kk, v)
+                runs = B.amskv_attended_tokens(c.h, layer, k)
+                den = torch.full((heads, len(runs)), float("nan"), dtype=torch.float64, device="cuda")
+                out = torch.full_like(q, float("nan"))
+                B.amskv_attend_density(c.h, layer, k, q, out, den, den.numel())
+                torch.cuda.synchronize()
+                tokens = [(s, t) for s, first, count in runs for t in range(first, first + count)]
+                want_out = oracle.attend_tokens(to_items(q), Ks, Vs, tokens, scale)
+                check_close(out, want_out, "output, layer %d scale %d" % (layer, k), max_abs=4e-2 if peaked else 1e-2)
+                want = oracle.attention_density(to_items(q), Ks, runs, scale, heads)
+                got = den.cpu().numpy()
+                assert np.allclose(got, want, rtol=2e-4, atol=1e-7), (layer, k, np.abs(got / want - 1).max())
+                counts = np.array([n for _, _, n in runs], dtype=np.float64)
+                assert np.allclose(got @ counts, sides[k] ** 2, rtol=1e-4)
+        assert B.amskv_status(c.h) == 0
