@@ -243,7 +243,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         // query rows a tile does not cover keep whatever the slot held before; start them at zero
         uint4* qz = reinterpret_cast<uint4*>(smem_raw + (q_smem - raw));
         for (uint32_t i = threadIdx.x; i < 2 * C::kQBytes / 16; i += C::kThreads) qz[i] = make_uint4(0, 0, 0, 0);
-        if (kDen) {
+        if constexpr (kDen) {
             uint4* dz = reinterpret_cast<uint4*>(smem_raw + (kv_smem - raw) + C::kStages * C::kStageBytes);
             for (uint32_t i = threadIdx.x; i < C::kDenBytes / 16; i += C::kThreads) dz[i] = make_uint4(0, 0, 0, 0);
         }
@@ -579,6 +579,8 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const uint32_t o_tmem = tmem + C::kOCol + g * D + lane_base;
         const uint32_t o_full = o_full0 + 8 * g;
         const bool q_loader = (wq == 0 && lane == 0);
+        // the output rows start on 32-byte boundaries (the interface only promises 16)
+        const bool o_sectors = ((reinterpret_cast<uintptr_t>(O) | (uintptr_t)(2 * o_row) | (uintptr_t)(2 * o_head) | (uintptr_t)(2 * o_tok)) & 31u) == 0;
         // density: [run][row] sums of this stream, in the shared memory the fourth key/value stage would take
         // (every thread only ever touches the entries of its own row; they were zeroed before the roles split)
         float* den_rows = reinterpret_cast<float*>(smem_raw + (kv_smem - raw) + C::kStages * C::kStageBytes) + g * kMaxDenRuns * kQRows;
@@ -765,15 +767,20 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     uint32_t o[32];
                     tmem_ld32(o_tmem + cblk * 32, o);
                     if (r < valid_rows) {
+                        uint32_t w[16];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint4 out4;
-                            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&out4);
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
+                            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        if (o_sectors) {
+                            // whole 32-byte sectors per thread: half the store instructions, no partly written sector
+                            st_global_32B(dst + cblk * 32, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                            st_global_32B(dst + cblk * 32 + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+                        } else {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                h[i] = __floats2bfloat162_rn(__uint_as_float(o[c * 8 + 2 * i]) * inv,
-                                                             __uint_as_float(o[c * 8 + 2 * i + 1]) * inv);
-                            reinterpret_cast<uint4*>(dst + cblk * 32)[c] = out4;
+                            for (int c = 0; c < 4; ++c)
+                                reinterpret_cast<uint4*>(dst + cblk * 32)[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
                         }
                     }
                 }
