@@ -717,29 +717,36 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                             }
                         }
                     }
-                    // P over S: columns 0..31 receive the 64 probabilities as bf16 pairs, 32 tokens per store
+                    // P over S: columns 0..31 receive the 64 probabilities as bf16 pairs, 16 tokens per store.
+                    // A partly filled tile only exponentiates the 16-token groups the products will read (the
+                    // P V is issued for as many 16-token steps): the columns behind them keep stale bits.
+                    int groups = kKT / 16;
+                    if (valid < kKT) groups = ((valid + 15) >> 4) + ((kExt && ext.rider_valid > 0 && j == n_tiles - 1) ? 1 : 0);
                     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t pk[kKT / 4];
+                    for (int grp = 0; grp < kKT / 16; ++grp) {
+                        if (grp < groups) {   // (the same for the whole warp)
+                            uint32_t pk[8];
 #pragma unroll
-                        for (int i = 0; i < kKT / 4; ++i) {
-                            const int c = half * (kKT / 2) + 2 * i;
-                            // every kPolyEvery-th pair takes its exponentials from a polynomial on the FMA pipe:
-                            // the special-function unit (16 results per clock per SM) is the narrowest resource
-                            float x0, x1, p0, p1;
-                            fma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), scale_log2, scale_log2, nb, nb);
-                            if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
-                                exp2_poly2(p0, p1, x0, x1);
-                            } else {
-                                p0 = fast_exp2(x0);
-                                p1 = fast_exp2(x1);
+                            for (int ii = 0; ii < 8; ++ii) {
+                                const int i = (grp & 1) * 8 + ii;   // pair index within its 32-token half, as before
+                                const int c = grp * 16 + 2 * ii;
+                                // every kPolyEvery-th pair takes its exponentials from a polynomial on the FMA pipe:
+                                // the special-function unit (16 results per clock per SM) is the narrowest resource
+                                float x0, x1, p0, p1;
+                                fma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), scale_log2, scale_log2, nb, nb);
+                                if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
+                                    exp2_poly2(p0, p1, x0, x1);
+                                } else {
+                                    p0 = fast_exp2(x0);
+                                    p1 = fast_exp2(x1);
+                                }
+                                add2(sum0, sum1, sum0, sum1, p0, p1);
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                                pk[ii] = *reinterpret_cast<const uint32_t*>(&h);
                             }
-                            add2(sum0, sum1, sum0, sum1, p0, p1);
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                            pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+                            tmem_st8_nowait(s_tmem + grp * 8, pk);
                         }
-                        tmem_st16_nowait(s_tmem + half * (kKT / 4), pk);
                     }
                     const float tile_sum = sum0 + sum1;
                     l += tile_sum;
