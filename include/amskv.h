@@ -81,9 +81,9 @@ extern "C" {
                                     (amskv_evicted_at). */
 
 /* amskv_set_attend_path */
-#define AMSKV_PATH_AUTO 0   /* CUDA-core kernel for a single query token, warp-per-item kernel for the
-                               other coarse scales (at most 16 queries and 32 retained keys), paired
-                               tcgen05 kernel otherwise                                             */
+#define AMSKV_PATH_AUTO 0   /* warp-per-item kernel for the coarse scales (at most 16 queries and 32
+                               retained keys; CUDA-core kernel for a single query token with several
+                               keys), paired tcgen05 kernel otherwise                               */
 #define AMSKV_PATH_SIMT 1   /* always the CUDA-core kernel                                     */
 #define AMSKV_PATH_TENSOR 2 /* always the single-stream tcgen05 kernel                         */
 #define AMSKV_PATH_TENSOR_PAIR 3 /* always the paired tcgen05 kernel (two query tiles per CTA)  */
@@ -210,10 +210,12 @@ AMSKV_API int amskv_attend(amskv_cache* cache, int layer, int scale, const void*
  * paired tensor-core kernel can read the scale's K and V from the caller's tensors, use them as
  * keys and values beside the older retained tokens it reads from the cache, and write them to
  * the scale's place in the cache on the way -- the separate copy and its second read of K and V
- * disappear.  Scales served by the other attention kernels, appends that are more than one
- * contiguous copy (a token budget whose ring wraps inside the scale) and, under AMSKV_PATH_AUTO,
- * scales of fewer than 64 tokens and scales where splitting the current scale off its cache range
- * would add a 64-token key tile, run as the two calls.
+ * disappear.  The warp-per-item kernel of the coarse scales does the same (it reads the scale's K and V
+ * from the caller's tensors and stores the registers that feed its products), and a single-token scale
+ * that is its own only key is one copy kernel (out = V).  Appends that are more than one contiguous copy
+ * (a token budget whose ring wraps inside the scale), scales served by the CUDA-core or the single-stream
+ * kernel and, under AMSKV_PATH_AUTO, paired-kernel scales of fewer than 64 tokens and scales where
+ * splitting the current scale off its cache range would add a 64-token key tile, run as the two calls.
  *   K, V: as for amskv_append (one stride triple kv_strides for both); Q, out: as for
  *   amskv_attend.  out must not overlap Q, K or V.
  * Stream ordering: as for the two calls -- this call must come after attend(layer, scale - 1)
