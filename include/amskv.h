@@ -214,7 +214,7 @@ AMSKV_API int amskv_attend(amskv_cache* cache, int layer, int scale, const void*
  * from the caller's tensors and stores the registers that feed its products), and a single-token scale
  * that is its own only key is one copy kernel (out = V).  Appends that are more than one contiguous copy
  * (a token budget whose ring wraps inside the scale), scales served by the CUDA-core or the single-stream
- * kernel and, under AMSKV_PATH_AUTO, paired-kernel scales of fewer than 64 tokens and scales where
+ * kernel and, under AMSKV_PATH_AUTO, paired-kernel scales of fewer than 32 tokens and scales where
  * splitting the current scale off its cache range would add a 64-token key tile, run as the two calls.
  *   K, V: as for amskv_append (one stride triple kv_strides for both); Q, out: as for
  *   amskv_attend.  out must not overlap Q, K or V.

@@ -485,9 +485,10 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
             return n;
         };
         if (tiles(ranges) + (T + 63) / 64 > tiles(after)) fused = false;
-        // Below a full key tile per scale the units are so short that the kernel is bound by the latency of
-        // its loads; holding a stage until it has been written out costs more there than the copy (measured).
-        if (T < 64) fused = false;
+        // Well below a full key tile per scale the units are so short that the kernel is bound by the latency of
+        // its loads; holding a stage until it has been written out costs as much there as the copy (measured:
+        // equal at T = 36, where fusing at least saves the launch and the second read; a loss at T = 25).
+        if (T < 32) fused = false;
     }
     if (!fused) {
         rc = amskv_append(cache, layer, scale, K, V, kv_strides, stream);
