@@ -80,6 +80,10 @@ extern "C" {
                                     scale as not retained (amskv_kept_segments) and as dropped at its own step
                                     (amskv_evicted_at). */
 
+#define AMSKV_FLAG_NVTX 8u /* amskv_append, amskv_attend and amskv_append_attend wrap their work in an NVTX range
+                              named after the call, layer and scale (timeline tools show which kernels belong to
+                              which step); no effect on results */
+
 /* amskv_set_attend_path */
 #define AMSKV_PATH_AUTO 0   /* warp-per-item kernel for the coarse scales (at most 16 queries and 32
                                retained keys; CUDA-core kernel for a single query token with several

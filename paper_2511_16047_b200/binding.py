@@ -22,6 +22,7 @@ MAX_SCALES = 32
 FLAG_PLAN_ONLY = 1
 FLAG_BULK_APPEND = 2
 FLAG_TRANSIENT_LAST_SCALE = 4
+FLAG_NVTX = 8
 PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_PAIR, PATH_SMALL = 0, 1, 2, 3, 4
 LAYER_EFFICIENT, LAYER_DEMANDING, LAYER_PROMOTABLE = 0, 1, 2
 

@@ -1,10 +1,13 @@
 // C ABI of the AMS-KV library: argument checking, the segment table and kernel launches.
 #include <atomic>
 #include <cmath>
+#include <cstdio>
 #include <cstring>
 #include <new>
 #include <numeric>
 #include <vector>
+
+#include <nvtx3/nvToolsExt.h>   // header-only; ranges cost nothing measurable unless a profiler is attached
 
 #include "../../include/amskv.h"
 #include "kernels.cuh"
@@ -61,6 +64,22 @@ struct amskv_cache {
 
 namespace {
 
+// A named range around one call's enqueueing, for timeline tools (cache flag AMSKV_FLAG_NVTX).
+struct CallRange {
+    bool on;
+    CallRange(const amskv_cache* c, const char* what, int layer, int scale) : on(c && (c->flags & AMSKV_FLAG_NVTX) != 0)
+    {
+        if (!on) return;
+        char name[64];
+        snprintf(name, sizeof(name), "%s L%d s%d", what, layer, scale);
+        nvtxRangePushA(name);
+    }
+    ~CallRange()
+    {
+        if (on) nvtxRangePop();
+    }
+};
+
 int check_desc(const amskv_desc* d)
 {
     if (!d || !d->scale_sides || !d->policy) return AMSKV_ERR_INVALID;
@@ -79,7 +98,7 @@ int check_desc(const amskv_desc* d)
         if (d->policy[l].n_condensed < 0 || d->policy[l].n_local < 1) return AMSKV_ERR_INVALID;
         if (d->policy[l].cache_demanding < 0 || d->policy[l].cache_demanding > AMSKV_LAYER_PROMOTABLE) return AMSKV_ERR_INVALID;
     }
-    if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND | AMSKV_FLAG_TRANSIENT_LAST_SCALE)) != 0)
+    if ((d->flags & ~(AMSKV_FLAG_PLAN_ONLY | AMSKV_FLAG_BULK_APPEND | AMSKV_FLAG_TRANSIENT_LAST_SCALE | AMSKV_FLAG_NVTX)) != 0)
         return AMSKV_ERR_INVALID;
     if (!(d->softmax_scale == d->softmax_scale)) return AMSKV_ERR_INVALID;  // NaN
     return AMSKV_OK;
@@ -287,6 +306,7 @@ int amskv_append(amskv_cache* cache, int layer, int scale, const void* K, const 
                  void* stream)
 {
     if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    const CallRange range(cache, "amskv_append", layer, scale);
     if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
     if (cache->transient(scale)) return AMSKV_ERR_UNSUPPORTED;   // it has no place in the arena: amskv_append_attend
     const int32_t T = cache->tokens[scale];
@@ -345,6 +365,7 @@ int amskv_attend(amskv_cache* cache, int layer, int scale, const void* Q, void* 
                  const int64_t o_strides[3], void* stream)
 {
     if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    const CallRange range(cache, "amskv_attend", layer, scale);
     if (cache->plan_only()) return AMSKV_ERR_UNSUPPORTED;
     if (scale != cache->last_appended[layer]) return AMSKV_ERR_ORDER;
     const int32_t T = cache->tokens[scale];
@@ -384,6 +405,7 @@ int amskv_append_attend(amskv_cache* cache, int layer, int scale, const void* K,
                         const int64_t o_strides[3], void* stream)
 {
     if (bad_layer_scale(cache, layer, scale)) return AMSKV_ERR_INVALID;
+    const CallRange range(cache, "amskv_append_attend", layer, scale);
     if (scale != cache->last_appended[layer] + 1) return AMSKV_ERR_ORDER;
     if (cache->plan_only()) {   // bookkeeping only
         note_appended(cache, layer, scale);

@@ -141,3 +141,18 @@ def test_broadcast_strides_are_refused():
         torch.cuda.synchronize()
         want = oracle.attend_selected(to_items(q), [to_items(k)], [to_items(v)], [0], 1.0 / math.sqrt(D))
         check_close(o, want, "one row, zero row stride")
+
+
+def test_nvtx_ranges_change_nothing():
+    """AMSKV_FLAG_NVTX wraps every call in a named range for timeline tools; outputs are bit-equal with and without."""
+    sides, rows, heads, D = (1, 2, 4, 9), 2, 3, 64
+    qkv = make_qkv(rows, heads, sides, D, seed=84)
+    with Cache(1, heads, D, rows, sides, [(1, 2, False)]) as a, Cache(1, heads, D, rows, sides, [(1, 2, False)], flags=B.FLAG_NVTX) as b:
+        for fused in (False, True):
+            oa, ob = run_pass(a, qkv, fused=fused), run_pass(b, qkv, fused=fused)
+            for x, y in zip(oa[0], ob[0]):
+                assert torch.equal(x, y)
+    d, keep = B.make_desc(1, heads, D, rows, sides, [(1, 2, False)], flags=16)
+    with pytest.raises(B.AmskvError) as e:
+        B.amskv_cache_create(d)
+    assert e.value.code == B.ERR_INVALID
