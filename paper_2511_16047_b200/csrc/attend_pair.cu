@@ -40,7 +40,7 @@ constexpr int kMmaWarp = 9;        // first MMA-issuing warp; Cfg<D>::kMmaWarps 
 constexpr int kMaxStages = 4;
 constexpr float kRescaleLog2 = 8.f;
 constexpr int kQSplitRows = 64;   // query tiles of at most this many rows are double-buffered inside their slot
-constexpr int kPolyEvery = 4;     // every 4th pair of exponentials goes to the FMA pipe (0: none)
+constexpr int kPolyEvery = 6;     // every 6th pair of exponentials goes to the FMA pipe (0: none); swept 2, 3, 4, 6, 8
 
 // kWide: one CTA per SM with two S buffers per stream and an issuing warp per stream (below): the form
 // 128 channels use.  64 channels use the two-CTA form (the wide form is instantiable for them, but lost
