@@ -37,10 +37,10 @@ FALLBACK_BF16_TFLOPS = 1400.0
 # `roofline.traffic` is then null.
 NCU_DOMINANT_KERNEL_TRAFFIC = {
     ("var_d30", "ams", "fused"): {
-        "bytes_per_launch": 2.001e9,
+        "bytes_per_launch": 1.655e9,
         "capture": "profiles/attention_dram_traffic_var_d30.md: 64-row, 2-layer case of the same shape, every launch of "
                    "attend_pair_kernel<64, ext> of one step, scaled by rows (x 8) and by the layers of each class (21 + 9), "
-                   "averaged over its 111 launches; reads exact, writes a lower bound (part of them still in L2 at that size)"},
+                   "averaged over its 141 launches; reads exact, writes a lower bound (part of them still in L2 at that size)"},
 }
 
 
@@ -64,7 +64,7 @@ def algorithmic_work(wl, policies, budgets=None, cache=None):
     from paper_2511_16047_b200 import binding as B
     items = wl.rows * wl.heads
     tok = wl.tokens
-    per = {}
+    per, keys = {}, {}
     for layer, (c, w, dem) in enumerate(policies):
         for k in range(len(tok)):
             if budgets is not None and budgets[layer][0] > 0:
@@ -72,7 +72,8 @@ def algorithmic_work(wl, policies, budgets=None, cache=None):
             else:
                 L = sum(tok[s] for s in _kept(k, c, w, dem))
             per[(layer, k)] = (2 * wl.head_dim * items * (2 * tok[k] + 2 * L), 4 * tok[k] * L * wl.head_dim * items)
-    return per
+            keys[(layer, k)] = L
+    return per, keys
 
 
 class ClockSampler:
@@ -186,7 +187,7 @@ def run_ours(args):
         cache = B.amskv_cache_create(desc, arena, nbytes)
         if args.path != "auto":
             B.amskv_set_attend_path(cache, {"simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR, "pair": B.PATH_TENSOR_PAIR, "small": B.PATH_SMALL}[args.path])
-        work = algorithmic_work(wl, policies, budgets, cache)
+        work, n_keys = algorithmic_work(wl, policies, budgets, cache)
 
         side = torch.cuda.Stream() if streams == 2 else None
         n_ev = wl.layers * K
@@ -319,7 +320,8 @@ def run_ours(args):
             result["pass_roofline_ms"] = sum(p["roofline_ms"] for p in per_scale)
             # the dominant kernel alone: the calls that ran as ONE launch of the paired kernel with the append
             # fused in (every launch of that kernel in a step, and nothing else, sits between their events)
-            dom = [key for key in work if one_launch[key]]
+            # (scales of at most 16 queries over at most 32 keys are the warp-per-item kernel's, not this one's)
+            dom = [key for key in work if one_launch[key] and (tok[key[1]] > 16 or n_keys[key] > 32)]
             if dom:
                 d_ms = sum(att_ms[key] for key in dom) / args.steps
                 d_bytes = sum(work[key][0] for key in dom)
