@@ -156,3 +156,19 @@ def test_nvtx_ranges_change_nothing():
     with pytest.raises(B.AmskvError) as e:
         B.amskv_cache_create(d)
     assert e.value.code == B.ERR_INVALID
+
+
+@pytest.mark.parametrize("fused", [False, True], ids=["separate", "fused"])
+def test_longest_schedule_many_ranges(fused):
+    """32 scales (the most a cache takes), a window of 7 and of 31 rotating slots: many short resident ranges per
+    call, every scale compared with the oracle."""
+    sides = tuple(1 + (i % 4) for i in range(B.MAX_SCALES))
+    rows, heads, D = 2, 3, 64
+    pols = [(3, 7, False), (0, 31, False), (5, 1, True)]
+    qkv = make_qkv(rows, heads, sides, D, seed=85)
+    with Cache(len(pols), heads, D, rows, sides, pols) as cache:
+        outs = run_pass(cache, qkv, fused=fused)
+        for layer, pol in enumerate(pols):
+            want = oracle_outputs(qkv, pol, 1.0 / math.sqrt(D))
+            for k in range(len(sides)):
+                check_close(outs[layer][k], want[k], "layer %d scale %d" % (layer, k))

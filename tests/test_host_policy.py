@@ -154,3 +154,25 @@ def test_compute_calls_fail_loudly_without_a_device():
     with pytest.raises(B.AmskvError) as e:
         B.amskv_cache_create(d)
     assert e.value.code == B.ERR_CUDA
+
+
+def test_longest_schedule_and_its_limits():
+    """AMSKV_MAX_SCALES scales are accepted (kept sets equal the oracle's at every step, window larger than a
+    handful of slots), one more is refused, and so are sides outside 1 .. 4096."""
+    import oracle
+    sides = tuple(1 + (i % 3) for i in range(B.MAX_SCALES))
+    pols = [(3, 7, False), (0, 31, False), (5, 1, True)]
+    d, keep = B.make_desc(len(pols), 2, 64, 2, sides, pols, flags=B.FLAG_PLAN_ONLY)
+    cache = B.amskv_cache_create(d)
+    for k in range(len(sides)):
+        for layer, (c, w, dem) in enumerate(pols):
+            assert B.lib.amskv_append(cache, layer, k, None, None, None, None) == B.OK
+            assert B.amskv_kept_segments(cache, layer, k) == oracle.keep_set(k, c, w, dem)
+            ranges = B.amskv_resident_ranges(cache, layer, k)
+            assert sum(n for _, n in ranges) == oracle.kept_tokens(sides, oracle.keep_set(k, c, w, dem))
+    B.amskv_cache_destroy(cache)
+    for bad in (sides + (1,), (0, 1), (1, 4097)):
+        d, keep = B.make_desc(1, 2, 64, 2, bad, [(1, 1, False)], flags=B.FLAG_PLAN_ONLY)
+        with pytest.raises(B.AmskvError) as e:
+            B.amskv_cache_create(d)
+        assert e.value.code == B.ERR_INVALID
