@@ -478,6 +478,18 @@ def run_ours(args):
                         "kernel_frac": round(dom["bytes_per_step"] / dom["ms_per_step"] / 1e6 / hbm_gbs, 4) if dom else None,
                         "kernel_timing": "CUDA events around each call in an eager replay of the same step",
                         "traffic": traffic, "traffic_note": traffic_note}
+        # Exponentials: one per (query, attended key) = flops / (4 D).  The special-function unit gives 16 per
+        # clock per SM (8.0 clocks per warp instruction per sub-partition, measured); with 64 channels it, not the
+        # tensor pipe, is the arithmetic floor (the tensor pipe needs 4 D / 8192 = 1/32 clock per exponential).
+        sm_mhz = (main["clocks"] or {}).get("sm_mhz") or 0
+        sm_count = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+        sfu_peak = 16.0 * sm_count * sm_mhz * 1e6 / 1e9   # G exponentials / s at the median clock of this run
+        exps = step_flops / (4.0 * wl.head_dim)
+        roofline["sfu"] = {"exps_per_step": exps, "achieved": round(exps / (ms / 1e3) / 1e9, 1),
+                           "peak": round(sfu_peak, 1) if sfu_peak else None, "unit": "Gexp/s",
+                           "frac": round(exps / (ms / 1e3) / 1e9 / sfu_peak, 4) if sfu_peak else None,
+                           "note": "all exponentials over 16 per clock per SM at the sampled median SM clock; "
+                                   "3 of 16 are computed by polynomial on the FMA pipe, so the unit itself sees 13/16 of this"}
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms, 4), "higher_is_better": False, "scaling": "weak",
