@@ -18,7 +18,10 @@
 // there is no shared-memory tile for P.  While one group exponentiates, the tensor pipe works
 // for the other.  The reference maximum of a row is the maximum of its first tile; O and the
 // row sum are rescaled only when a later tile exceeds it by more than 2^8, so for
-// well-conditioned logits they are never touched.  The first lane of each group fetches its
+// well-conditioned logits they are never touched.  Launches of three key tiles or more (kLazy)
+// do not even take the later tiles' maxima: a tile is exponentiated against the reference as it
+// stands, and only a row whose tile sum leaves the range (beyond 2^64, or not a number) makes
+// its warp take the true maxima, rescale and form the tile again.  The first lane of each group fetches its
 // next query tile as soon as the last S of the current one has landed.
 // Every wait is bounded: a wait that gives up records a status code, all roles wind down,
 // copies in flight are awaited and the tensor memory is freed.
@@ -40,6 +43,7 @@ constexpr int kMmaWarp = 9;        // first MMA-issuing warp; Cfg<D>::kMmaWarps 
 constexpr int kMaxStages = 4;
 constexpr float kRescaleLog2 = 8.f;
 constexpr int kQSplitRows = 64;   // query tiles of at most this many rows are double-buffered inside their slot
+constexpr float kLazySumLimit = 1.8446744e19f;   // 2^64: see the kLazy form of the softmax loop
 constexpr int kPolyEvery = 6;     // every 6th pair of exponentials goes to the FMA pipe (0: none); swept 2, 3, 4, 6, 8
 
 // kWide: one CTA per SM with two S buffers per stream and an issuing warp per stream (below): the form
@@ -189,7 +193,7 @@ __device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0,
 }
 
 // ---------------------------------------------------------------- kernel
-template <int D, bool kExt, bool kWide, bool kDen>
+template <int D, bool kExt, bool kWide, bool kDen, bool kLazy>
 __global__ void __launch_bounds__(Cfg<D, kWide, kDen>::kThreads, Cfg<D, kWide, kDen>::kCtasPerSm)
 attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap k_map64,
@@ -666,55 +670,63 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                             if ((((i < 32 ? keep_lo : keep_hi) >> (i & 31)) & 1u) == 0u) sr[i] = 0xff800000u;  // -inf
                     }
                     // row maximum with four independent chains
-                    float mx[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        mx[c] = max3(__uint_as_float(sr[c]), __uint_as_float(sr[4 + c]), __uint_as_float(sr[8 + c]));
-#pragma unroll
-                    for (int i = 12; i < kKT - 4; i += 8) {
+                    auto row_max = [&]() -> float {
+                        float mx[4];
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            mx[c] = max3(mx[c], __uint_as_float(sr[i + c]), __uint_as_float(sr[i + 4 + c]));
-                    }
+                            mx[c] = max3(__uint_as_float(sr[c]), __uint_as_float(sr[4 + c]), __uint_as_float(sr[8 + c]));
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(sr[kKT - 4 + c]));
-                    const float mt = fmaxf(max3(mx[0], mx[1], mx[2]), mx[3]);
+                        for (int i = 12; i < kKT - 4; i += 8) {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                mx[c] = max3(mx[c], __uint_as_float(sr[i + c]), __uint_as_float(sr[i + 4 + c]));
+                        }
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(sr[kKT - 4 + c]));
+                        return fmaxf(max3(mx[0], mx[1], mx[2]), mx[3]);
+                    };
+                    // rare: bring O and the row sum to a new reference (rows with `grow`).  The previous P V must
+                    // be done.  One S buffer: it was issued before this tile's S, whose arrival covers every
+                    // earlier product.  Two buffers: this S may have been issued first, so wait for the
+                    // product's own completion (one arrival per P V; at most one phase can be ahead,
+                    // because the next P V needs the P this tile has not written yet).
+                    auto rescale = [&](const bool grow, const float mt) -> bool {
+                        if (C::kSBufs == 2 && !__all_sync(0xffffffffu, mbar_wait(pv_done0 + 8 * g, (t - 1u) & 1u, abort_flag))) {
+                            report(status, kStatusSyncTimeout, abort_flag);
+                            return false;
+                        }
+                        if (C::kSBufs == 2) tc_fence_after();
+                        float alpha = 1.f;
+                        if (grow) {
+                            alpha = fast_exp2((m_ref - mt) * scale_log2);
+                            m_ref = mt;
+                            nb = -mt * scale_log2;
+                            l *= alpha;
+                            if (kDen) {
+                                run_mass *= alpha;
+                                for (int rn = 0; rn < den.n_runs; ++rn) den_rows[rn * kQRows + r] *= alpha;
+                            }
+                        }
+#pragma unroll 1
+                        for (int cblk = 0; cblk < D / 8; ++cblk) {
+                            uint32_t o[8];
+                            tmem_ld8(o_tmem + cblk * 8, o);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st8(o_tmem + cblk * 8, o);
+                        }
+                        return true;
+                    };
                     if (j == 0) {
+                        const float mt = row_max();
                         m_ref = mt;
                         nb = -mt * scale_log2;
-                    } else {
+                    } else if (!kLazy) {
+                        const float mt = row_max();
                         const bool grow = fmaf(mt, scale_log2, nb) > kRescaleLog2;
-                        if (__any_sync(0xffffffffu, grow)) {
-                            // rare: bring O and the row sum to the new reference.  The previous P V must be done.
-                            // One S buffer: it was issued before this tile's S, whose arrival covers every
-                            // earlier product.  Two buffers: this S may have been issued first, so wait for the
-                            // product's own completion (one arrival per P V; at most one phase can be ahead,
-                            // because the next P V needs the P this tile has not written yet).
-                            if (C::kSBufs == 2 && !__all_sync(0xffffffffu, mbar_wait(pv_done0 + 8 * g, (t - 1u) & 1u, abort_flag))) {
-                                report(status, kStatusSyncTimeout, abort_flag);
-                                ok = false;
-                                break;
-                            }
-                            if (C::kSBufs == 2) tc_fence_after();
-                            float alpha = 1.f;
-                            if (grow) {
-                                alpha = fast_exp2((m_ref - mt) * scale_log2);
-                                m_ref = mt;
-                                nb = -mt * scale_log2;
-                                l *= alpha;
-                                if (kDen) {
-                                    run_mass *= alpha;
-                                    for (int rn = 0; rn < den.n_runs; ++rn) den_rows[rn * kQRows + r] *= alpha;
-                                }
-                            }
-#pragma unroll 1
-                            for (int cblk = 0; cblk < D / 8; ++cblk) {
-                                uint32_t o[8];
-                                tmem_ld8(o_tmem + cblk * 8, o);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                                tmem_st8(o_tmem + cblk * 8, o);
-                            }
+                        if (__any_sync(0xffffffffu, grow) && !rescale(grow, mt)) {
+                            ok = false;
+                            break;
                         }
                     }
                     // P over S: columns 0..31 receive the 64 probabilities as bf16 pairs, 16 tokens per store.
@@ -722,33 +734,55 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     // P V is issued for as many 16-token steps): the columns behind them keep stale bits.
                     int groups = kKT / 16;
                     if (valid < kKT) groups = ((valid + 15) >> 4) + ((kExt && ext.rider_valid > 0 && j == n_tiles - 1) ? 1 : 0);
-                    float sum0 = 0.f, sum1 = 0.f;
+                    auto exp_tile = [&]() -> float {
+                        float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                    for (int grp = 0; grp < kKT / 16; ++grp) {
-                        if (grp < groups) {   // (the same for the whole warp)
-                            uint32_t pk[8];
+                        for (int grp = 0; grp < kKT / 16; ++grp) {
+                            if (grp < groups) {   // (the same for the whole warp)
+                                uint32_t pk[8];
 #pragma unroll
-                            for (int ii = 0; ii < 8; ++ii) {
-                                const int i = (grp & 1) * 8 + ii;   // pair index within its 32-token half, as before
-                                const int c = grp * 16 + 2 * ii;
-                                // every kPolyEvery-th pair takes its exponentials from a polynomial on the FMA pipe:
-                                // the special-function unit (16 results per clock per SM) is the narrowest resource
-                                float x0, x1, p0, p1;
-                                fma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), scale_log2, scale_log2, nb, nb);
-                                if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
-                                    exp2_poly2(p0, p1, x0, x1);
-                                } else {
-                                    p0 = fast_exp2(x0);
-                                    p1 = fast_exp2(x1);
+                                for (int ii = 0; ii < 8; ++ii) {
+                                    const int i = (grp & 1) * 8 + ii;   // pair index within its 32-token half, as before
+                                    const int c = grp * 16 + 2 * ii;
+                                    // every kPolyEvery-th pair takes its exponentials from a polynomial on the FMA pipe:
+                                    // the special-function unit (16 results per clock per SM) is the narrowest resource
+                                    float x0, x1, p0, p1;
+                                    fma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), scale_log2, scale_log2, nb, nb);
+                                    if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
+                                        exp2_poly2(p0, p1, x0, x1);
+                                    } else {
+                                        p0 = fast_exp2(x0);
+                                        p1 = fast_exp2(x1);
+                                    }
+                                    add2(sum0, sum1, sum0, sum1, p0, p1);
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                                    pk[ii] = *reinterpret_cast<const uint32_t*>(&h);
                                 }
-                                add2(sum0, sum1, sum0, sum1, p0, p1);
-                                const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                                pk[ii] = *reinterpret_cast<const uint32_t*>(&h);
+                                tmem_st8_nowait(s_tmem + grp * 8, pk);
                             }
-                            tmem_st8_nowait(s_tmem + grp * 8, pk);
+                        }
+                        return sum0 + sum1;
+                    };
+                    float tile_sum = exp_tile();
+                    if (kLazy && j > 0) {
+                        // No maximum was taken for this tile: its exponentials were formed against the row's reference
+                        // as it stood (the maximum of the unit's first tile, or of the last tile that was redone).
+                        // That is exact as long as nothing overflows.  A row whose tile sum is beyond the limit (or
+                        // not a number) has outgrown its reference by more than 2^58; the warp then takes the tile's
+                        // true maxima, rescales and forms the tile again before it announces P.  The polynomial
+                        // saturates at 2^126, so it cannot hide such a row.
+                        const bool over = !(tile_sum <= kLazySumLimit);
+                        if (__any_sync(0xffffffffu, over)) {
+                            tmem_wait_st();
+                            const float mt = row_max();
+                            const bool grow = over || fmaf(mt, scale_log2, nb) > kRescaleLog2;
+                            if (!rescale(grow, mt)) {
+                                ok = false;
+                                break;
+                            }
+                            tile_sum = exp_tile();
                         }
                     }
-                    const float tile_sum = sum0 + sum1;
                     l += tile_sum;
                     if (kDen) run_mass += tile_sum;
                     tmem_wait_st();
@@ -830,7 +864,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 }
 
 // ---------------------------------------------------------------- host side
-template <int D, bool kExt, bool kWide, bool kDen>
+template <int D, bool kExt, bool kWide, bool kDen, bool kLazy>
 cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& km64,
                    const CUtensorMap& vm64, const ExtArgs& ext, const Strided& O,
                    const RangeList& ranges, int32_t T, int32_t heads, const PairPlan& pp, int32_t n_tiles, int3 qpos,
@@ -838,11 +872,11 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
 {
     using C = Cfg<D, kWide, kDen>;
     static SharedMemoryOptIn opt_in;
-    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide, kDen>, (int)C::kSmemBytes);
+    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide, kDen, kLazy>, (int)C::kSmemBytes);
     if (oe != cudaSuccess) return oe;
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > pp.n_pairs) grid = pp.n_pairs;
-    attend_pair_kernel<D, kExt, kWide, kDen><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
+    attend_pair_kernel<D, kExt, kWide, kDen, kLazy><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
         qm, km, vm, km64, vm64, ext, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos,
         scale_log2, status, den);
     count_launch();
@@ -923,17 +957,29 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     // 64 channels always take the two-CTA form: the wide form was measured on the tensor-bound launches of a
     // 2 240-token schedule (T = 576 and 1 024, 36 heads) and lost there too (26.3 vs 20.8 and 64.2 vs 53.9 ms):
     // two streams per SM do not keep the tensor pipe as busy as four, even with the chain broken.
-#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE, DEN)                                                                        \
-    return launch<DD, EXT, WIDE, DEN>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos, scale_log2,   \
-                                      status, sm_count, stream, den)
+#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE, DEN, LAZY)                                                                  \
+    return launch<DD, EXT, WIDE, DEN, LAZY>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos,         \
+                                            scale_log2, status, sm_count, stream, den)
+    // Launches of three key tiles or more take the row maximum of a unit's first tile only (the kLazy form of the
+    // softmax loop: 1.7 % of a 256x256-shaped pass, 6 % of a 1024x1024-shaped one); with fewer tiles there is next
+    // to nothing to skip and the plain form is the faster code.
+    constexpr int lazy_min = 3, lazy128_min = 3;
     if (D == 128) {
-        if (density) AMSKV_PAIR_LAUNCH(128, false, true, true);
-        if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false);
-        AMSKV_PAIR_LAUNCH(128, false, true, false);
+        if (density) AMSKV_PAIR_LAUNCH(128, false, true, true, false);
+        if (n_tiles >= lazy128_min) {
+            if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false, true);
+            AMSKV_PAIR_LAUNCH(128, false, true, false, true);
+        }
+        if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false, false);
+        AMSKV_PAIR_LAUNCH(128, false, true, false, false);
     }
-    if (density) AMSKV_PAIR_LAUNCH(64, false, false, true);
-    if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false);
-    AMSKV_PAIR_LAUNCH(64, false, false, false);
+    if (density) AMSKV_PAIR_LAUNCH(64, false, false, true, false);
+    if (n_tiles >= lazy_min) {
+        if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, true);
+        AMSKV_PAIR_LAUNCH(64, false, false, false, true);
+    }
+    if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, false);
+    AMSKV_PAIR_LAUNCH(64, false, false, false, false);
 #undef AMSKV_PAIR_LAUNCH
 }
 

@@ -272,12 +272,12 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, f
 // 2^x for a pair on the FMA pipe instead of the special-function unit: x = n + f with n the
 // nearest integer (obtained by adding 1.5 * 2^23), 2^f by a cubic on [-0.5, 0.5] (relative error
 // below 1e-3, under the bf16 rounding the result gets anyway), and n added into the exponent
-// field.  Inputs below -127 (including -inf) give exactly 0.
+// field.  Inputs below -127 (including -inf) give exactly 0; inputs above 126 give 2^126.
 __device__ __forceinline__ void exp2_poly2(float& y0, float& y1, float x0, float x1)
 {
     constexpr float kMagic = 12582912.f;   // 1.5 * 2^23
-    x0 = fmaxf(x0, -127.f);
-    x1 = fmaxf(x1, -127.f);
+    x0 = fminf(fmaxf(x0, -127.f), 126.f);
+    x1 = fminf(fmaxf(x1, -127.f), 126.f);
     float r0, r1, n0, n1, f0, f1, p0, p1;
     add2(r0, r1, x0, x1, kMagic, kMagic);
     add2(n0, n1, r0, r1, -kMagic, -kMagic);

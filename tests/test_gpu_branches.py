@@ -43,17 +43,20 @@ def test_peaked_softmax_rows_head_dim_128(path, fused):
 @pytest.mark.parametrize("fused", [False, True], ids=["separate", "fused"])
 @pytest.mark.parametrize("path", ["pair", "auto", "tensor", "simt"])
 @pytest.mark.parametrize("D", [64, 128])
-def test_reference_maximum_moves_in_every_key_tile(D, path, fused):
-    """Keys built so that every row's largest logit grows by 8 (11.5 in base-2 units, above the kernels'
-    rescale threshold of 2^8) from one 64-token tile to the next: the accumulator and the row sum are
-    brought to a new reference in every tile of every row, several times per work unit."""
+@pytest.mark.parametrize("step", [8, 48])
+def test_reference_maximum_moves_in_every_key_tile(D, path, fused, step):
+    """Keys built so that every row's largest logit grows by `step` from one 64-token tile to the next.
+    step 8 (11.5 in base-2 units, above the rescale threshold of 2^8): a kernel that takes every tile's
+    maximum brings the accumulator and the row sum to a new reference in every tile of every row.
+    step 48 (69 in base-2 units, above the 2^64 limit on a tile's sum): a kernel that only takes the first
+    tile's maximum finds every later tile out of range and has to form each of them a second time."""
     _need(D)
     sides = (8, 18)                      # 64 + 324 keys: seven key tiles at the last scale, three query tiles
     rows, heads = 3, 5
     scale = 1.0 / 8 if D == 64 else 1.0 / 16
     qkv, level = [], 0
     for k, s in enumerate(sides):
-        qkv.append(synth.growing_logit_qkv(rows, heads, s * s, D, 82, k, first_level=level, device="cuda"))
+        qkv.append(synth.growing_logit_qkv(rows, heads, s * s, D, 82, k, first_level=level, step=step, device="cuda"))
         level += (s * s + 63) // 64
     # the inputs do what they are meant to: per-tile maxima of the true logits climb by more than 2^8 (base 2)
     q, kk = to_items(qkv[1][0])[0], np.concatenate([to_items(qkv[0][1])[0], to_items(qkv[1][1])[0]], 0)
