@@ -193,7 +193,7 @@ __device__ __forceinline__ void tile_at(const RangeList& rl, int j, int32_t& t0,
 }
 
 // ---------------------------------------------------------------- kernel
-template <int D, bool kExt, bool kWide, bool kDen, bool kLazy>
+template <int D, bool kExt, bool kWide, bool kDen, bool kLazy, bool kShort>
 __global__ void __launch_bounds__(Cfg<D, kWide, kDen>::kThreads, Cfg<D, kWide, kDen>::kCtasPerSm)
 attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap k_map64,
@@ -310,6 +310,22 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         // requested (it has landed by then, so the wait costs nothing), by lane 0, as one bulk group per
         // stage; before a stage is refilled, every group but the two newest has finished reading it.
         const bool storing = kExt && ext.store != 0;
+        if (kShort && lane == 0) {
+            prefetch_tensormap(&k_map);
+            prefetch_tensormap(&v_map);
+            prefetch_tensormap(&k_map64);
+            prefetch_tensormap(&v_map64);
+            if (kExt) {
+                prefetch_tensormap(&ext.k64);
+                prefetch_tensormap(&ext.v64);
+                prefetch_tensormap(&ext.k16);
+                prefetch_tensormap(&ext.v16);
+                if (storing) {
+                    prefetch_tensormap(&ext.k_store);
+                    prefetch_tensormap(&ext.v_store);
+                }
+            }
+        }
         uint32_t st_sq[2] = {0, 0};
         int32_t st_tok[2] = {0, 0}, st_item[2] = {0, 0};
         int st_n = 0;
@@ -365,23 +381,18 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     }
                     const uint32_t full = kv_full0 + 8 * stage;
                     const uint32_t k_dst = kv_smem + stage * C::kStageBytes, v_dst = k_dst + C::kKVBytes;
-                    if (elect_one()) {
-                        mbar_expect_tx(full, (uint32_t)(nch + (rider ? 1 : 0)) * kKVBoxRows * D * 2 * 2);
-                        if (rider) {
-#pragma unroll
-                            for (int h = 0; h < C::kHalves; ++h) {
-                                tma_load_3d(k_dst + h * C::kKVHalfBytes + nch * kKVBoxRows * 128, &k_map, full, h * 64,
-                                            ext.rider_tok, item);
-                                tma_load_3d(v_dst + h * C::kKVHalfBytes + nch * kKVBoxRows * 128, &v_map, full, h * 64,
-                                            ext.rider_tok, item);
-                            }
-                        }
-                        if (from_ext) {
-                            const int32_t row = item / heads, head = item - row * heads;
-                            int c[4] = {0, 0, 0, 0};
-                            c[ext.pos.y] = head;
-                            c[ext.pos.z] = row;
-                            if (nch == kKT / kKVBoxRows) {
+                    // A tile of the caller's tensors that no rider shares its stage with is one 64-token box whatever
+                    // its length: the tokens past the end of the scale are outside the tensor, cost no traffic and
+                    // arrive as zeros (the products never read their rows, the fused write is clipped at the scale's end).
+                    const bool whole_box = nch == kKT / kKVBoxRows || (kShort && from_ext && !rider);
+                    if (whole_box) {
+                        if (elect_one()) {
+                            mbar_expect_tx(full, (uint32_t)kKT * D * 2 * 2);
+                            if (from_ext) {
+                                const int32_t row = item / heads, head = item - row * heads;
+                                int c[4] = {0, 0, 0, 0};
+                                c[ext.pos.y] = head;
+                                c[ext.pos.z] = row;
                                 c[ext.pos.x] = t0;
 #pragma unroll
                                 for (int h = 0; h < C::kHalves; ++h) {
@@ -389,6 +400,31 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                                     tma_load_4d(v_dst + h * C::kKVHalfBytes, &ext.v64, full, h * 64, c[1], c[2], c[3]);
                                 }
                             } else {
+#pragma unroll
+                                for (int h = 0; h < C::kHalves; ++h) {
+                                    tma_load_3d(k_dst + h * C::kKVHalfBytes, &k_map64, full, h * 64, t0, item);
+                                    tma_load_3d(v_dst + h * C::kKVHalfBytes, &v_map64, full, h * 64, t0, item);
+                                }
+                            }
+                        }
+                    } else if (!kShort) {
+                        // 16-token boxes (and the rider's box), issued by one lane
+                        if (elect_one()) {
+                            mbar_expect_tx(full, (uint32_t)(nch + (rider ? 1 : 0)) * kKVBoxRows * D * 2 * 2);
+                            if (rider) {
+#pragma unroll
+                                for (int h = 0; h < C::kHalves; ++h) {
+                                    tma_load_3d(k_dst + h * C::kKVHalfBytes + nch * kKVBoxRows * 128, &k_map, full, h * 64,
+                                                ext.rider_tok, item);
+                                    tma_load_3d(v_dst + h * C::kKVHalfBytes + nch * kKVBoxRows * 128, &v_map, full, h * 64,
+                                                ext.rider_tok, item);
+                                }
+                            }
+                            if (from_ext) {
+                                const int32_t row = item / heads, head = item - row * heads;
+                                int c[4] = {0, 0, 0, 0};
+                                c[ext.pos.y] = head;
+                                c[ext.pos.z] = row;
                                 for (int bx = 0; bx < nch; ++bx) {
                                     c[ext.pos.x] = t0 + bx * kKVBoxRows;
 #pragma unroll
@@ -399,22 +435,39 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                                                     c[1], c[2], c[3]);
                                     }
                                 }
-                            }
-                        } else if (nch == kKT / kKVBoxRows) {
+                            } else {
+                                for (int bx = 0; bx < nch; ++bx) {
 #pragma unroll
-                            for (int h = 0; h < C::kHalves; ++h) {
-                                tma_load_3d(k_dst + h * C::kKVHalfBytes, &k_map64, full, h * 64, t0, item);
-                                tma_load_3d(v_dst + h * C::kKVHalfBytes, &v_map64, full, h * 64, t0, item);
-                            }
-                        } else {
-                            for (int bx = 0; bx < nch; ++bx) {
-#pragma unroll
-                                for (int h = 0; h < C::kHalves; ++h) {
-                                    tma_load_3d(k_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &k_map, full, h * 64,
-                                                t0 + bx * kKVBoxRows, item);
-                                    tma_load_3d(v_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &v_map, full, h * 64,
-                                                t0 + bx * kKVBoxRows, item);
+                                    for (int h = 0; h < C::kHalves; ++h) {
+                                        tma_load_3d(k_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &k_map, full, h * 64,
+                                                    t0 + bx * kKVBoxRows, item);
+                                        tma_load_3d(v_dst + h * C::kKVHalfBytes + bx * kKVBoxRows * 128, &v_map, full, h * 64,
+                                                    t0 + bx * kKVBoxRows, item);
+                                    }
                                 }
+                            }
+                        }
+                    } else {
+                        // Short units (at most four key tiles): one lane per bulk copy, all issued by one instruction.  A
+                        // lane issuing six or eight copies one after the other is what such units wait for (the issuing
+                        // warp of a 36-token scale spent half its time waiting for tiles).
+                        if (lane == 0) mbar_expect_tx(full, (uint32_t)(nch + (rider ? 1 : 0)) * kKVBoxRows * D * 2 * 2);
+                        __syncwarp();
+                        const int n_main = 2 * C::kHalves * nch, n_ops = n_main + (rider ? 2 * C::kHalves : 0);
+                        if (lane < n_ops) {
+                            const bool is_rider = lane >= n_main;
+                            const int o = is_rider ? lane - n_main : lane;
+                            const int h = o % C::kHalves, kv = (o / C::kHalves) & 1, bx = is_rider ? nch : o / (2 * C::kHalves);
+                            const uint32_t dst = (kv ? v_dst : k_dst) + h * C::kKVHalfBytes + bx * kKVBoxRows * 128;
+                            if (from_ext && !is_rider) {
+                                const int32_t row = item / heads, head = item - row * heads;
+                                int c[4] = {0, 0, 0, 0};
+                                c[ext.pos.y] = head;
+                                c[ext.pos.z] = row;
+                                c[ext.pos.x] = t0 + bx * kKVBoxRows;
+                                tma_load_4d(dst, kv ? &ext.v16 : &ext.k16, full, h * 64, c[1], c[2], c[3]);
+                            } else {
+                                tma_load_3d(dst, kv ? &v_map : &k_map, full, h * 64, is_rider ? ext.rider_tok : t0 + bx * kKVBoxRows, item);
                             }
                         }
                     }
@@ -592,6 +645,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         uint32_t q_next_n = 0;    // first pair index not yet searched for a query tile
 
         // request the query tile of this stream's next unit not yet requested (first lane of the group only)
+        if (kShort && q_loader) prefetch_tensormap(&q_map);
         auto load_next_q = [&]() {
             for (; q_next_n < my_pairs; ++q_next_n) {
                 const int32_t pair = (int32_t)(blockIdx.x + q_next_n * gridDim.x);
@@ -864,7 +918,7 @@ attend_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 }
 
 // ---------------------------------------------------------------- host side
-template <int D, bool kExt, bool kWide, bool kDen, bool kLazy>
+template <int D, bool kExt, bool kWide, bool kDen, bool kLazy, bool kShort>
 cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& km64,
                    const CUtensorMap& vm64, const ExtArgs& ext, const Strided& O,
                    const RangeList& ranges, int32_t T, int32_t heads, const PairPlan& pp, int32_t n_tiles, int3 qpos,
@@ -872,11 +926,11 @@ cudaError_t launch(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorM
 {
     using C = Cfg<D, kWide, kDen>;
     static SharedMemoryOptIn opt_in;
-    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide, kDen, kLazy>, (int)C::kSmemBytes);
+    const cudaError_t oe = opt_in.ensure(attend_pair_kernel<D, kExt, kWide, kDen, kLazy, kShort>, (int)C::kSmemBytes);
     if (oe != cudaSuccess) return oe;
     int64_t grid = (int64_t)sm_count * C::kCtasPerSm;
     if (grid > pp.n_pairs) grid = pp.n_pairs;
-    attend_pair_kernel<D, kExt, kWide, kDen, kLazy><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
+    attend_pair_kernel<D, kExt, kWide, kDen, kLazy, kShort><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
         qm, km, vm, km64, vm64, ext, (__nv_bfloat16*)O.ptr, O.row, O.head, O.token, ranges, T, heads, pp, n_tiles, qpos,
         scale_log2, status, den);
     count_launch();
@@ -957,29 +1011,36 @@ cudaError_t launch_attend_pair(const Strided& Q, const Strided& O, const void* k
     // 64 channels always take the two-CTA form: the wide form was measured on the tensor-bound launches of a
     // 2 240-token schedule (T = 576 and 1 024, 36 heads) and lost there too (26.3 vs 20.8 and 64.2 vs 53.9 ms):
     // two streams per SM do not keep the tensor pipe as busy as four, even with the chain broken.
-#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE, DEN, LAZY)                                                                  \
-    return launch<DD, EXT, WIDE, DEN, LAZY>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos,         \
-                                            scale_log2, status, sm_count, stream, den)
+#define AMSKV_PAIR_LAUNCH(DD, EXT, WIDE, DEN, LAZY, SHORT)                                                          \
+    return launch<DD, EXT, WIDE, DEN, LAZY, SHORT>(qm, km, vm, km64, vm64, ext, O, ranges, T, heads, pp, n_tiles, qpos,  \
+                                                   scale_log2, status, sm_count, stream, den)
     // Launches of three key tiles or more take the row maximum of a unit's first tile only (the kLazy form of the
     // softmax loop: 1.7 % of a 256x256-shaped pass, 6 % of a 1024x1024-shaped one); with fewer tiles there is next
-    // to nothing to skip and the plain form is the faster code.
-    constexpr int lazy_min = 3, lazy128_min = 3;
+    // to nothing to skip and the plain form is the faster code.  Launches of at most four key tiles (kShort, 64
+    // channels) have a producer that issues a tile's bulk copies from several lanes at once and fetches a partly
+    // filled tile of the caller's tensors as one box; the long launches keep the one-lane producer (its smaller code
+    // measured 2 % faster there).
+    constexpr int lazy_min = 3, lazy128_min = 3, short_max = 4;
     if (D == 128) {
-        if (density) AMSKV_PAIR_LAUNCH(128, false, true, true, false);
+        if (density) AMSKV_PAIR_LAUNCH(128, false, true, true, false, false);
         if (n_tiles >= lazy128_min) {
-            if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false, true);
-            AMSKV_PAIR_LAUNCH(128, false, true, false, true);
+            if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false, true, false);
+            AMSKV_PAIR_LAUNCH(128, false, true, false, true, false);
         }
-        if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false, false);
-        AMSKV_PAIR_LAUNCH(128, false, true, false, false);
+        if (cur) AMSKV_PAIR_LAUNCH(128, true, true, false, false, false);
+        AMSKV_PAIR_LAUNCH(128, false, true, false, false, false);
     }
-    if (density) AMSKV_PAIR_LAUNCH(64, false, false, true, false);
+    if (density) AMSKV_PAIR_LAUNCH(64, false, false, true, false, false);
+    if (n_tiles > short_max) {
+        if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, true, false);
+        AMSKV_PAIR_LAUNCH(64, false, false, false, true, false);
+    }
     if (n_tiles >= lazy_min) {
-        if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, true);
-        AMSKV_PAIR_LAUNCH(64, false, false, false, true);
+        if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, true, true);
+        AMSKV_PAIR_LAUNCH(64, false, false, false, true, true);
     }
-    if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, false);
-    AMSKV_PAIR_LAUNCH(64, false, false, false, false);
+    if (cur) AMSKV_PAIR_LAUNCH(64, true, false, false, false, true);
+    AMSKV_PAIR_LAUNCH(64, false, false, false, false, true);
 #undef AMSKV_PAIR_LAUNCH
 }
 
